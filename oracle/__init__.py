@@ -1,0 +1,201 @@
+"""ctypes front end of the CPU oracle (`dmr_oracle.c`).
+
+TEST INFRASTRUCTURE ONLY. The product path never imports this package; only the tests, the
+smoke check and the benchmark's CPU-baseline leg do. It shares nothing with the CUDA
+library: it compiles its own C file with gcc and works on numpy arrays.
+
+All tensors are numpy arrays: bf16 tensors are uint16 bit patterns, outputs are float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dmr_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+OK = 0
+ERR_ARG = 1
+ERR_NONFINITE = 5
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, no FMA contraction, OpenMP). Returns the .so path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-std=c11", "-O2", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def _L():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_bf16_to_f64.restype = ctypes.c_double
+        _lib.oracle_bf16_to_f64.argtypes = [ctypes.c_uint16]
+        _lib.oracle_f64_to_bf16_rne.restype = ctypes.c_uint16
+        _lib.oracle_f64_to_bf16_rne.argtypes = [ctypes.c_double]
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code):
+        super().__init__(f"oracle error code {code}")
+        self.code = code
+
+
+def _check(code):
+    if code != OK:
+        raise OracleError(code)
+
+
+def num_threads() -> int:
+    return int(_L().oracle_num_threads())
+
+
+def group_of(K: int, group: int) -> int:
+    return K if group == 0 else group
+
+
+def f64_to_bf16_rne(x: float) -> int:
+    return int(_L().oracle_f64_to_bf16_rne(float(x)))
+
+
+def bf16_to_f64(b: int) -> float:
+    return float(_L().oracle_bf16_to_f64(int(b)))
+
+
+def pack(codes: np.ndarray, bits: int) -> np.ndarray:
+    codes = _c(codes, np.uint8)
+    N, K = codes.shape
+    out = np.zeros((N, K * bits // 32), dtype=np.uint32)
+    _check(_L().oracle_pack(_p(codes), N, K, bits, _p(out)))
+    return out
+
+
+def unpack(qweight: np.ndarray, K: int, bits: int) -> np.ndarray:
+    qweight = _c(qweight, np.uint32)
+    N = qweight.shape[0]
+    out = np.zeros((N, K), dtype=np.uint8)
+    _check(_L().oracle_unpack(_p(qweight), N, K, bits, _p(out)))
+    return out
+
+
+def quantize(W: np.ndarray, bits: int = 4, group: int = 128, return_codes: bool = False):
+    """W [N][K] bf16 bits -> (qweight u32 [N][K*bits/32], scales u16 [N][G], zeros u8 [N][G])."""
+    W = _c(W, np.uint16)
+    N, K = W.shape
+    g = group_of(K, group)
+    if K % g != 0 or K % (32 // bits) != 0:
+        raise OracleError(ERR_ARG)
+    G = K // g
+    qweight = np.zeros((N, K * bits // 32), dtype=np.uint32)
+    scales = np.zeros((N, G), dtype=np.uint16)
+    zeros = np.zeros((N, G), dtype=np.uint8)
+    codes = np.zeros((N, K), dtype=np.uint8) if return_codes else None
+    _check(_L().oracle_quantize(_p(W), N, K, bits, group, _p(qweight), _p(scales), _p(zeros), _p(codes)))
+    if return_codes:
+        return qweight, scales, zeros, codes
+    return qweight, scales, zeros
+
+
+def dequantize(qweight, scales, zeros, K: int, bits: int = 4, group: int = 128):
+    """-> (What float64 [N][K] exact s*(q-z), What_bf16 u16 [N][K] nearest bf16)."""
+    qweight = _c(qweight, np.uint32)
+    scales = _c(scales, np.uint16)
+    zeros = _c(zeros, np.uint8)
+    N = qweight.shape[0]
+    What = np.zeros((N, K), dtype=np.float64)
+    Wb = np.zeros((N, K), dtype=np.uint16)
+    _check(_L().oracle_dequantize(_p(qweight), _p(scales), _p(zeros), N, K, bits, group, _p(What), _p(Wb)))
+    return What, Wb
+
+
+def lowbit_linear(X, qweight, scales, zeros, bits: int = 4, group: int = 128, rounded: bool = False):
+    """Y [M][N] float64 = X . dequant(Wq)^T (rounded=True uses the nearest-bf16 dequantized weights)."""
+    X = _c(X, np.uint16)
+    qweight = _c(qweight, np.uint32)
+    scales = _c(scales, np.uint16)
+    zeros = _c(zeros, np.uint8)
+    M, K = X.shape
+    N = qweight.shape[0]
+    Y = np.zeros((M, N), dtype=np.float64)
+    _check(_L().oracle_lowbit_linear(_p(X), M, _p(qweight), _p(scales), _p(zeros), N, K, bits, group,
+                                     int(rounded), _p(Y)))
+    return Y
+
+
+def dense_linear(X, W):
+    X = _c(X, np.uint16)
+    W = _c(W, np.uint16)
+    M, K = X.shape
+    N = W.shape[0]
+    Y = np.zeros((M, N), dtype=np.float64)
+    _check(_L().oracle_dense_linear(_p(X), M, _p(W), N, K, _p(Y)))
+    return Y
+
+
+def routed_linear(X, mask, W, qweight, scales, zeros, bits: int = 4, group: int = 128):
+    X = _c(X, np.uint16)
+    mask = _c(mask, np.uint8)
+    W = _c(W, np.uint16)
+    qweight = _c(qweight, np.uint32)
+    scales = _c(scales, np.uint16)
+    zeros = _c(zeros, np.uint8)
+    M, K = X.shape
+    N = W.shape[0]
+    Y = np.zeros((M, N), dtype=np.float64)
+    _check(_L().oracle_routed_linear(_p(X), M, _p(mask), _p(W), _p(qweight), _p(scales), _p(zeros),
+                                     N, K, bits, group, _p(Y)))
+    return Y
+
+
+def sampled_linear(X, ms, ns, *, mask=None, W=None, qweight=None, scales=None, zeros=None,
+                   bits: int = 4, group: int = 128, rounded: bool = False):
+    """Values of the (routed / low-bit / dense) linear at the output coordinates (ms[i], ns[i])."""
+    X = _c(X, np.uint16)
+    M, K = X.shape
+    ms = _c(ms, np.int32)
+    ns = _c(ns, np.int32)
+    if W is not None:
+        W = _c(W, np.uint16)
+        N = W.shape[0]
+    if qweight is not None:
+        qweight = _c(qweight, np.uint32)
+        scales = _c(scales, np.uint16)
+        zeros = _c(zeros, np.uint8)
+        N = qweight.shape[0]
+    if mask is not None:
+        mask = _c(mask, np.uint8)
+    out = np.zeros(len(ms), dtype=np.float64)
+    _check(_L().oracle_sampled_linear(_p(X), M, _p(mask), _p(W), _p(qweight), _p(scales), _p(zeros),
+                                      N, K, bits, group, int(rounded), _p(ms), _p(ns), len(ms), _p(out)))
+    return out
+
+
+def route_partition(mask):
+    mask = _c(mask, np.uint8)
+    M = mask.shape[0]
+    ih = np.zeros(max(M, 1), dtype=np.int32)
+    il = np.zeros(max(M, 1), dtype=np.int32)
+    nh = ctypes.c_int32(0)
+    nl = ctypes.c_int32(0)
+    _check(_L().oracle_route_partition(_p(mask), M, _p(ih), _p(il), ctypes.byref(nh), ctypes.byref(nl)))
+    return ih[:nh.value].copy(), il[:nl.value].copy()
