@@ -1,0 +1,155 @@
+/*
+ * libdmr: low-bit and step-routed decoder linear layers for Dynamic Mixed-Precision Routing,
+ * written for NVIDIA B200 (sm_100a).  Plain C ABI: pointers and sizes only.
+ *
+ * The operations follow the paper's problem statement:
+ *   - Sec. 3 (Problem Formulation): a set of LLMs derived from one base model under different
+ *     numerical precisions; a routing index r_t chosen per step (Eq. 1) selects which precision
+ *     serves that step.
+ *   - Sec. 5 "Experimental Models and Precision" and App. "Quantization Detail": the
+ *     low-precision model is W4A16 weight-only quantization of every decoder Linear layer
+ *     (activations stay 16 bit); the high-precision reference is bf16.
+ *   - Sec. 4.2 "KL-to-Classification Mapping": label 1 means the step needs high precision.
+ * The paper fixes no quantization arithmetic; the scheme implemented here is round-to-nearest
+ * asymmetric min/max quantization with an integer zero point and a bf16 scale per group of
+ * consecutive input features (see dmr_quantize).
+ *
+ * Conventions
+ *   W  [N][K] bf16, row-major (N = out features, K = in features, like a Linear weight)
+ *   X  [M][K] bf16, row-major (M = tokens, or concurrent agent steps)
+ *   Y  [M][N] bf16 or fp32, row-major
+ *   qweight [N][K*bits/32] uint32.  bits = 4: code k of a row is in word k/8, bits 4*(k%8)..+3.
+ *                                   bits = 8: code k is in word k/4, bits 8*(k%4)..+7.
+ *                                   Codes are unsigned, 0 .. 2^bits-1.
+ *   scales  [N][G] bf16, zeros [N][G] uint8, G = K / g, g = group_size (0 means g = K).
+ *   Dequantized weight: scale * (code - zero).
+ *
+ * Unless a parameter says "host", every data pointer is a DEVICE pointer owned by the caller.
+ * The library allocates no device memory.  `stream` is a cudaStream_t passed as void*; all work
+ * is enqueued on it and no call synchronises the host.  Argument errors are reported before
+ * anything is launched.  Pointers must be 16-byte aligned.
+ */
+#ifndef DMR_H_
+#define DMR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DMR_OK = 0,
+    DMR_ERR_INVALID_ARG = 1, /* null pointer, negative size, K not a multiple of the group ... */
+    DMR_ERR_UNSUPPORTED = 2, /* a format or shape this build has no kernel for */
+    DMR_ERR_ALIGNMENT = 3,   /* a pointer is not 16-byte aligned */
+    DMR_ERR_WORKSPACE = 4,   /* workspace is NULL or smaller than dmr_workspace_bytes() */
+    DMR_ERR_NONFINITE = 5,   /* written to dev_status by dmr_quantize: NaN/Inf weight seen */
+    DMR_ERR_TIMEOUT = 6,     /* written to the workspace status word: a bounded wait ran out */
+    DMR_ERR_CUDA = 7         /* a CUDA call failed; see dmr_last_cuda_error() */
+} dmr_status_t;
+
+typedef struct {
+    int32_t bits;       /* 4 or 8 */
+    int32_t group_size; /* 64, 128, ... (multiple of 32, divides K), or 0 = one group per row */
+} dmr_qformat_t;
+
+typedef enum { DMR_OUT_BF16 = 0, DMR_OUT_F32 = 1 } dmr_out_t;
+
+typedef enum {
+    DMR_OP_LOWBIT_LINEAR = 0,
+    DMR_OP_DENSE_LINEAR = 1,
+    DMR_OP_ROUTED_LINEAR = 2
+} dmr_op_t;
+
+/* Sizes of the quantized tensors in bytes (0 if the format is invalid for K). */
+size_t dmr_qweight_bytes(int N, int K, dmr_qformat_t f);
+size_t dmr_scales_bytes(int N, int K, dmr_qformat_t f);
+size_t dmr_zeros_bytes(int N, int K, dmr_qformat_t f);
+
+/* Scratch bytes `op` needs for these sizes (split-K partial sums, routed row lists and
+ * compacted activations, a status word).  Always a multiple of 256; never 0. */
+size_t dmr_workspace_bytes(dmr_op_t op, int M, int N, int K, dmr_qformat_t f);
+
+/*
+ * Quantize and pack bf16 weights (the low-precision model of Sec. 5 / App. "Quantization
+ * Detail": weight-only, 16-bit activations).  Per row n and group j of g consecutive k, in
+ * binary64, with qmax = 2^bits - 1:
+ *   lo = min(0, min w), hi = max(0, max w);  s = nearest bf16 to (hi - lo) / qmax (ties to
+ *   even; 1.0 for an all-zero group; raised to 2^-126 if it would be zero or subnormal);
+ *   zero = clamp(rint(-lo / s), 0, qmax);  code_k = clamp(rint(w_k / s) + zero, 0, qmax).
+ * Outputs: qweight, scales, zeros as laid out above.  dev_status: one int32 on the device,
+ * set to DMR_ERR_NONFINITE if any weight is NaN or Inf (outputs are then unspecified) and
+ * left untouched otherwise; the caller zeroes it beforehand.  May be NULL.
+ * Requires K % g == 0, g % 32 == 0, K % 32 == 0.
+ */
+dmr_status_t dmr_quantize(const void *W_bf16, int N, int K, dmr_qformat_t f, void *qweight,
+                          void *scales, void *zeros, int32_t *dev_status, void *stream);
+
+/* Test utility: W_out[n][k] = scale * (code - zero), as fp32 (exact) or bf16 (nearest). */
+dmr_status_t dmr_dequantize(const void *qweight, const void *scales, const void *zeros, int N,
+                            int K, dmr_qformat_t f, void *W_out, dmr_out_t out, void *stream);
+
+/*
+ * Low-precision linear layer (the W4A16 model's Linear, Sec. 5): Y = X . dequant(Wq)^T with fp32
+ * accumulation.  M <= 16 runs the bandwidth-bound decode kernel, larger M the tensor-core GEMM.
+ * M = 0 is a no-op.  workspace: dmr_workspace_bytes(DMR_OP_LOWBIT_LINEAR, ...) bytes.
+ */
+dmr_status_t dmr_lowbit_linear(const void *X_bf16, int M, const void *qweight, const void *scales,
+                               const void *zeros, int N, int K, dmr_qformat_t f, void *Y,
+                               dmr_out_t out, void *workspace, size_t workspace_bytes,
+                               void *stream);
+
+/* High-precision linear layer (the bf16 reference model, Sec. 5): Y = X . W^T, fp32 accumulation. */
+dmr_status_t dmr_dense_linear(const void *X_bf16, int M, const void *W_bf16, int N, int K, void *Y,
+                              dmr_out_t out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Step-routed linear layer (Sec. 3, Eq. 1: the router picks a precision per step; Sec. 4.2:
+ * label 1 = high precision).  mask [M] uint8 on the device: rows with mask != 0 are multiplied
+ * with the bf16 weights W, the others with the low-bit weights; every row's result is written
+ * at its own index m, so Y is in step order.  The mask is read on the device only.  Row m equals,
+ * bit for bit, row m of dmr_dense_linear (mask != 0) or dmr_lowbit_linear (mask == 0) called
+ * on the same M rows.
+ */
+dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, const void *W_bf16,
+                               const void *qweight, const void *scales, const void *zeros, int N,
+                               int K, dmr_qformat_t f, void *Y, dmr_out_t out, void *workspace,
+                               size_t workspace_bytes, void *stream);
+
+/*
+ * Stable partition of step indices by mask (the split that dmr_routed_linear performs first).
+ * idx_high / idx_low: int32 [M] each; counts: int32 [2] = {n_high, n_low}.  All on the device.
+ */
+dmr_status_t dmr_route_partition(const uint8_t *mask, int M, int32_t *idx_high, int32_t *idx_low,
+                                 int32_t *counts, void *stream);
+
+/*
+ * dmr_lowbit_linear for callers whose activations live in host memory: X_host [M][K] bf16 and
+ * Y_host [M][N] are HOST pointers (pinned memory makes the copies asynchronous); the weights stay
+ * on the device.  The call copies X to the device, runs the layer and copies Y back, all on
+ * `stream`, and returns without synchronising.  staging: device scratch of
+ * dmr_host_staging_bytes(M, N, K, out) bytes.
+ */
+size_t dmr_host_staging_bytes(int M, int N, int K, dmr_out_t out);
+dmr_status_t dmr_lowbit_linear_host(const void *X_host, int M, const void *qweight,
+                                    const void *scales, const void *zeros, int N, int K,
+                                    dmr_qformat_t f, void *Y_host, dmr_out_t out, void *staging,
+                                    size_t staging_bytes, void *workspace, size_t workspace_bytes,
+                                    void *stream);
+
+/* Reads the status word a previous call may have set in `workspace` (DMR_OK or DMR_ERR_TIMEOUT).
+ * Synchronises `stream`. */
+dmr_status_t dmr_workspace_status(const void *workspace, void *stream);
+
+const char *dmr_status_string(dmr_status_t s);
+int dmr_last_cuda_error(void);
+
+/* Number of kernels this library has launched in this process (for launch accounting). */
+uint64_t dmr_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DMR_H_ */

@@ -1,0 +1,249 @@
+"""ctypes binding of libdmr.so: argument marshalling only, every step runs in the CUDA kernels.
+
+Functions carry the names of the C entry points (include/dmr.h) and take torch CUDA tensors
+(or, for the *_host call, pinned host tensors). There is no CPU fallback: if the library is
+missing or a call fails, a DmrError is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libdmr.so")
+
+OUT_BF16 = 0
+OUT_F32 = 1
+OP_LOWBIT, OP_DENSE, OP_ROUTED = 0, 1, 2
+
+
+class DmrError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"libdmr: {msg} (status {code})")
+        self.code = code
+
+
+class QFormat(ctypes.Structure):
+    """dmr_qformat_t: bits in {4, 8}; group_size 0 = one group per output row."""
+    _fields_ = [("bits", ctypes.c_int32), ("group_size", ctypes.c_int32)]
+
+    def group(self, K: int) -> int:
+        return K if self.group_size == 0 else self.group_size
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libdmr.so (built in-tree by paper_2602_02711_b200.build). Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise DmrError(-1, f"{_LIB_PATH} not found: run `python -m paper_2602_02711_b200.build`")
+    L = ctypes.CDLL(_LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    for name in ("dmr_qweight_bytes", "dmr_scales_bytes", "dmr_zeros_bytes"):
+        getattr(L, name).restype = sz
+        getattr(L, name).argtypes = [i32, i32, QFormat]
+    L.dmr_workspace_bytes.restype = sz
+    L.dmr_workspace_bytes.argtypes = [i32, i32, i32, i32, QFormat]
+    L.dmr_quantize.restype = i32
+    L.dmr_quantize.argtypes = [vp, i32, i32, QFormat, vp, vp, vp, vp, vp]
+    L.dmr_dequantize.restype = i32
+    L.dmr_dequantize.argtypes = [vp, vp, vp, i32, i32, QFormat, vp, i32, vp]
+    L.dmr_lowbit_linear.restype = i32
+    L.dmr_lowbit_linear.argtypes = [vp, i32, vp, vp, vp, i32, i32, QFormat, vp, i32, vp, sz, vp]
+    L.dmr_dense_linear.restype = i32
+    L.dmr_dense_linear.argtypes = [vp, i32, vp, i32, i32, vp, i32, vp, sz, vp]
+    L.dmr_routed_linear.restype = i32
+    L.dmr_routed_linear.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, i32, QFormat, vp, i32, vp, sz, vp]
+    L.dmr_route_partition.restype = i32
+    L.dmr_route_partition.argtypes = [vp, i32, vp, vp, vp, vp]
+    L.dmr_host_staging_bytes.restype = sz
+    L.dmr_host_staging_bytes.argtypes = [i32, i32, i32, i32]
+    L.dmr_lowbit_linear_host.restype = i32
+    L.dmr_lowbit_linear_host.argtypes = [vp, i32, vp, vp, vp, i32, i32, QFormat, vp, i32, vp, sz, vp, sz, vp]
+    L.dmr_workspace_status.restype = i32
+    L.dmr_workspace_status.argtypes = [vp, vp]
+    L.dmr_status_string.restype = ctypes.c_char_p
+    L.dmr_status_string.argtypes = [i32]
+    L.dmr_last_cuda_error.restype = i32
+    L.dmr_launch_count.restype = ctypes.c_uint64
+    _lib = L
+    return L
+
+
+def _check(code: int):
+    if code != 0:
+        L = lib()
+        msg = L.dmr_status_string(code).decode()
+        if code == 7:
+            msg += f" (cudaError {L.dmr_last_cuda_error()})"
+        raise DmrError(code, msg)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str):
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise DmrError(1, f"{name} must be a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def dmr_launch_count() -> int:
+    return int(lib().dmr_launch_count())
+
+
+def dmr_workspace_bytes(op: int, M: int, N: int, K: int, fmt: QFormat) -> int:
+    return int(lib().dmr_workspace_bytes(op, M, N, K, fmt))
+
+
+def new_workspace(op: int, M: int, N: int, K: int, fmt: QFormat, device="cuda") -> torch.Tensor:
+    """A zeroed scratch buffer of the size `op` needs (torch owns the memory)."""
+    return torch.zeros(dmr_workspace_bytes(op, M, N, K, fmt), dtype=torch.uint8, device=device)
+
+
+@dataclass
+class QuantizedLinear:
+    """Packed weights of one Linear layer as dmr_quantize lays them out."""
+    qweight: torch.Tensor  # int32 [N][K*bits/32]
+    scales: torch.Tensor   # bf16  [N][G]
+    zeros: torch.Tensor    # uint8 [N][G]
+    N: int
+    K: int
+    fmt: QFormat
+
+    def weight_bytes(self) -> int:
+        return self.qweight.numel() * 4 + self.scales.numel() * 2 + self.zeros.numel()
+
+
+def dmr_quantize(W: torch.Tensor, fmt: QFormat, stream=None, check: bool = True) -> QuantizedLinear:
+    """bf16 W [N][K] -> packed codes + per-group scale / zero. check=True synchronises to read the status."""
+    _dev(W, torch.bfloat16, "W")
+    N, K = W.shape
+    L = lib()
+    qb = L.dmr_qweight_bytes(N, K, fmt)
+    if qb == 0:
+        raise DmrError(1, "invalid quantization format for this K")
+    G = K // fmt.group(K)
+    qweight = torch.empty((N, K * fmt.bits // 32), dtype=torch.int32, device=W.device)
+    scales = torch.empty((N, G), dtype=torch.bfloat16, device=W.device)
+    zeros = torch.empty((N, G), dtype=torch.uint8, device=W.device)
+    status = torch.zeros(1, dtype=torch.int32, device=W.device)
+    _check(L.dmr_quantize(_ptr(W), N, K, fmt, _ptr(qweight), _ptr(scales), _ptr(zeros), _ptr(status), _stream(stream)))
+    if check:
+        code = int(status.item())
+        if code != 0:
+            _check(code)
+    return QuantizedLinear(qweight, scales, zeros, N, K, fmt)
+
+
+def quantize_layer(W: torch.Tensor, bits: int = 4, group_size: int = 128) -> QuantizedLinear:
+    return dmr_quantize(W, QFormat(bits, group_size))
+
+
+def dmr_dequantize(q: QuantizedLinear, out: int = OUT_F32, stream=None) -> torch.Tensor:
+    W = torch.empty((q.N, q.K), dtype=torch.float32 if out == OUT_F32 else torch.bfloat16, device=q.qweight.device)
+    _check(lib().dmr_dequantize(_ptr(q.qweight), _ptr(q.scales), _ptr(q.zeros), q.N, q.K, q.fmt, _ptr(W), out,
+                                _stream(stream)))
+    return W
+
+
+def _out_tensor(M, N, out, device, Y):
+    dt = torch.float32 if out == OUT_F32 else torch.bfloat16
+    if Y is None:
+        return torch.empty((M, N), dtype=dt, device=device)
+    return _dev(Y, dt, "Y")
+
+
+def dmr_lowbit_linear(X: torch.Tensor, q: QuantizedLinear, out: int = OUT_BF16, Y=None, workspace=None,
+                      stream=None) -> torch.Tensor:
+    """Y = X . dequant(Wq)^T."""
+    _dev(X, torch.bfloat16, "X")
+    M, K = X.shape
+    if K != q.K:
+        raise DmrError(1, "X and the quantized weights disagree on K")
+    Y = _out_tensor(M, q.N, out, X.device, Y)
+    if workspace is None:
+        workspace = new_workspace(OP_LOWBIT, M, q.N, K, q.fmt, X.device)
+    _check(lib().dmr_lowbit_linear(_ptr(X), M, _ptr(q.qweight), _ptr(q.scales), _ptr(q.zeros), q.N, K, q.fmt,
+                                   _ptr(Y), out, _ptr(workspace), workspace.numel(), _stream(stream)))
+    return Y
+
+
+def dmr_dense_linear(X: torch.Tensor, W: torch.Tensor, out: int = OUT_BF16, Y=None, workspace=None,
+                     stream=None) -> torch.Tensor:
+    """Y = X . W^T with bf16 weights."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(W, torch.bfloat16, "W")
+    M, K = X.shape
+    N = W.shape[0]
+    if W.shape[1] != K:
+        raise DmrError(1, "X and W disagree on K")
+    Y = _out_tensor(M, N, out, X.device, Y)
+    if workspace is None:
+        workspace = new_workspace(OP_DENSE, M, N, K, QFormat(4, 0), X.device)
+    _check(lib().dmr_dense_linear(_ptr(X), M, _ptr(W), N, K, _ptr(Y), out, _ptr(workspace), workspace.numel(),
+                                  _stream(stream)))
+    return Y
+
+
+def dmr_routed_linear(X: torch.Tensor, mask: torch.Tensor, W: torch.Tensor, q: QuantizedLinear,
+                      out: int = OUT_BF16, Y=None, workspace=None, stream=None) -> torch.Tensor:
+    """Rows with mask != 0 use the bf16 weights, the others the low-bit weights; Y keeps step order."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(W, torch.bfloat16, "W")
+    _dev(mask, torch.uint8, "mask")
+    M, K = X.shape
+    if mask.numel() != M or W.shape != (q.N, K) or q.K != K:
+        raise DmrError(1, "shape mismatch")
+    Y = _out_tensor(M, q.N, out, X.device, Y)
+    if workspace is None:
+        workspace = new_workspace(OP_ROUTED, M, q.N, K, q.fmt, X.device)
+    _check(lib().dmr_routed_linear(_ptr(X), M, _ptr(mask), _ptr(W), _ptr(q.qweight), _ptr(q.scales), _ptr(q.zeros),
+                                   q.N, K, q.fmt, _ptr(Y), out, _ptr(workspace), workspace.numel(), _stream(stream)))
+    return Y
+
+
+def dmr_route_partition(mask: torch.Tensor, stream=None):
+    """-> (idx_high int32 [M], idx_low int32 [M], counts int32 [2] = {n_high, n_low}), all on the device."""
+    _dev(mask, torch.uint8, "mask")
+    M = mask.numel()
+    ih = torch.empty(max(M, 1), dtype=torch.int32, device=mask.device)
+    il = torch.empty(max(M, 1), dtype=torch.int32, device=mask.device)
+    counts = torch.empty(2, dtype=torch.int32, device=mask.device)
+    _check(lib().dmr_route_partition(_ptr(mask), M, _ptr(ih), _ptr(il), _ptr(counts), _stream(stream)))
+    return ih, il, counts
+
+
+def dmr_lowbit_linear_host(X_host: torch.Tensor, q: QuantizedLinear, Y_host: torch.Tensor, out: int = OUT_BF16,
+                           staging=None, workspace=None, stream=None):
+    """Host-buffer variant: X_host / Y_host are (pinned) CPU tensors; copies run on `stream`."""
+    if X_host.is_cuda or Y_host.is_cuda:
+        raise DmrError(1, "X_host and Y_host must be CPU tensors")
+    M, K = X_host.shape
+    L = lib()
+    dev = q.qweight.device
+    if staging is None:
+        staging = torch.empty(L.dmr_host_staging_bytes(M, q.N, K, out), dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = new_workspace(OP_LOWBIT, M, q.N, K, q.fmt, dev)
+    _check(L.dmr_lowbit_linear_host(_ptr(X_host), M, _ptr(q.qweight), _ptr(q.scales), _ptr(q.zeros), q.N, K, q.fmt,
+                                    _ptr(Y_host), out, _ptr(staging), staging.numel(), _ptr(workspace),
+                                    workspace.numel(), _stream(stream)))
+    return Y_host

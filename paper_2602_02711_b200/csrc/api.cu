@@ -1,0 +1,276 @@
+// C ABI of libdmr: argument validation, kernel-family choice and workspace carving.
+// Every entry point validates first and launches afterwards; nothing here synchronises the host
+// except dmr_workspace_status.
+#include <cstring>
+
+#include "common.cuh"
+
+namespace dmr {
+int g_last_cuda_error = 0;
+unsigned long long g_launches = 0;
+
+namespace {
+
+struct RoutedWs {
+    int32_t *counts;    // {n_high, n_low}
+    int32_t *idx_high;  // [Mpad]
+    int32_t *idx_low;   // [Mpad]
+    size_t end;         // bytes used from the workspace base
+};
+
+size_t routed_lists_bytes(int M) { return 256 + 2 * round_up((size_t)(M > 0 ? M : 1) * 4, 256); }
+
+RoutedWs carve_routed(void *workspace, int M) {
+    char *base = reinterpret_cast<char *>(workspace) + kWsStatusBytes;
+    const size_t list = round_up((size_t)(M > 0 ? M : 1) * 4, 256);
+    RoutedWs w;
+    w.counts = reinterpret_cast<int32_t *>(base);
+    w.idx_high = reinterpret_cast<int32_t *>(base + 256);
+    w.idx_low = reinterpret_cast<int32_t *>(base + 256 + list);
+    w.end = kWsStatusBytes + 256 + 2 * list;
+    return w;
+}
+
+dmr_status_t common_checks(const void *X, int M, int N, int K, const void *Y, dmr_out_t out) {
+    if (M < 0 || N < 1 || K < 1) return DMR_ERR_INVALID_ARG;
+    if (out != DMR_OUT_BF16 && out != DMR_OUT_F32) return DMR_ERR_INVALID_ARG;
+    if (M > 0 && (!X || !Y)) return DMR_ERR_INVALID_ARG;
+    if (!aligned16(X) || !aligned16(Y)) return DMR_ERR_ALIGNMENT;
+    if (K % 8 != 0) return DMR_ERR_UNSUPPORTED;  // rows must be 16-byte multiples
+    return DMR_OK;
+}
+
+// Rows [0, M) (sel.idx == null) or the listed rows, low-bit weights.  Chooses the kernel family
+// from (M, N, K, format) only, never from how many rows a routed call found.
+dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales,
+                        const uint8_t *zeros, int N, int K, dmr_qformat_t f, void *Y, dmr_out_t out,
+                        cudaStream_t st) {
+    const int g = group_of(K, f);
+    const size_t ysz = out == DMR_OUT_F32 ? 4 : 2;
+    if (!decode_lowbit_supported(M < 16 ? M : 16, N, K, f.bits, g))
+        return launch_simple_lowbit(X, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, st);
+    for (int m0 = 0; m0 < M; m0 += 16) {
+        const int mc = M - m0 < 16 ? M - m0 : 16;
+        RowSel s = sel;
+        const uint16_t *Xc = X;
+        void *Yc = Y;
+        if (sel.idx) {
+            s.idx = sel.idx + m0;
+            s.offset = sel.offset + m0;
+        } else {
+            Xc = X + (size_t)m0 * K;
+            Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
+        }
+        dmr_status_t r = launch_decode_lowbit(Xc, mc, s, qweight, scales, zeros, N, K, f.bits, g, Yc, out, st);
+        if (r != DMR_OK) return r;
+    }
+    return DMR_OK;
+}
+
+dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N, int K, void *Y,
+                       dmr_out_t out, cudaStream_t st) {
+    const size_t ysz = out == DMR_OUT_F32 ? 4 : 2;
+    if (!decode_dense_supported(M < 16 ? M : 16, N, K)) return launch_simple_dense(X, M, sel, W, N, K, Y, out, st);
+    for (int m0 = 0; m0 < M; m0 += 16) {
+        const int mc = M - m0 < 16 ? M - m0 : 16;
+        RowSel s = sel;
+        const uint16_t *Xc = X;
+        void *Yc = Y;
+        if (sel.idx) {
+            s.idx = sel.idx + m0;
+            s.offset = sel.offset + m0;
+        } else {
+            Xc = X + (size_t)m0 * K;
+            Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
+        }
+        dmr_status_t r = launch_decode_dense(Xc, mc, s, W, N, K, Yc, out, st);
+        if (r != DMR_OK) return r;
+    }
+    return DMR_OK;
+}
+
+}  // namespace
+}  // namespace dmr
+
+using namespace dmr;
+
+extern "C" {
+
+size_t dmr_qweight_bytes(int N, int K, dmr_qformat_t f) {
+    if (N < 1 || !format_ok(K, f)) return 0;
+    return (size_t)N * K * f.bits / 8;
+}
+
+size_t dmr_scales_bytes(int N, int K, dmr_qformat_t f) {
+    if (N < 1 || !format_ok(K, f)) return 0;
+    return (size_t)N * (K / group_of(K, f)) * 2;
+}
+
+size_t dmr_zeros_bytes(int N, int K, dmr_qformat_t f) {
+    if (N < 1 || !format_ok(K, f)) return 0;
+    return (size_t)N * (K / group_of(K, f));
+}
+
+size_t dmr_workspace_bytes(dmr_op_t op, int M, int N, int K, dmr_qformat_t f) {
+    (void)N;
+    (void)K;
+    (void)f;
+    size_t b = kWsStatusBytes;
+    if (op == DMR_OP_ROUTED_LINEAR) b += routed_lists_bytes(M);
+    return round_up(b, 256);
+}
+
+dmr_status_t dmr_quantize(const void *W_bf16, int N, int K, dmr_qformat_t f, void *qweight, void *scales,
+                          void *zeros, int32_t *dev_status, void *stream) {
+    if (N < 1 || K < 1 || !W_bf16 || !qweight || !scales || !zeros) return DMR_ERR_INVALID_ARG;
+    if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
+    if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
+    if (!aligned16(W_bf16) || !aligned16(qweight)) return DMR_ERR_ALIGNMENT;
+    return launch_quantize(reinterpret_cast<const uint16_t *>(W_bf16), N, K, f.bits, group_of(K, f),
+                           reinterpret_cast<uint32_t *>(qweight), reinterpret_cast<uint16_t *>(scales),
+                           reinterpret_cast<uint8_t *>(zeros), dev_status, (cudaStream_t)stream);
+}
+
+dmr_status_t dmr_dequantize(const void *qweight, const void *scales, const void *zeros, int N, int K,
+                            dmr_qformat_t f, void *W_out, dmr_out_t out, void *stream) {
+    if (N < 1 || K < 1 || !qweight || !scales || !zeros || !W_out) return DMR_ERR_INVALID_ARG;
+    if (out != DMR_OUT_BF16 && out != DMR_OUT_F32) return DMR_ERR_INVALID_ARG;
+    if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
+    if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
+    if (!aligned16(qweight) || !aligned16(W_out)) return DMR_ERR_ALIGNMENT;
+    return launch_dequantize(reinterpret_cast<const uint32_t *>(qweight), reinterpret_cast<const uint16_t *>(scales),
+                             reinterpret_cast<const uint8_t *>(zeros), N, K, f.bits, group_of(K, f), W_out, out,
+                             (cudaStream_t)stream);
+}
+
+dmr_status_t dmr_lowbit_linear(const void *X_bf16, int M, const void *qweight, const void *scales,
+                               const void *zeros, int N, int K, dmr_qformat_t f, void *Y, dmr_out_t out,
+                               void *workspace, size_t workspace_bytes, void *stream) {
+    dmr_status_t r = common_checks(X_bf16, M, N, K, Y, out);
+    if (r != DMR_OK) return r;
+    if (!qweight || !scales || !zeros) return DMR_ERR_INVALID_ARG;
+    if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
+    if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
+    if (!aligned16(qweight)) return DMR_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < dmr_workspace_bytes(DMR_OP_LOWBIT_LINEAR, M, N, K, f)) return DMR_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
+    if (M == 0) return DMR_OK;
+    RowSel sel = {nullptr, nullptr, 0};
+    return run_lowbit(reinterpret_cast<const uint16_t *>(X_bf16), M, sel, reinterpret_cast<const uint32_t *>(qweight),
+                      reinterpret_cast<const uint16_t *>(scales), reinterpret_cast<const uint8_t *>(zeros), N, K, f,
+                      Y, out, (cudaStream_t)stream);
+}
+
+dmr_status_t dmr_dense_linear(const void *X_bf16, int M, const void *W_bf16, int N, int K, void *Y,
+                              dmr_out_t out, void *workspace, size_t workspace_bytes, void *stream) {
+    dmr_status_t r = common_checks(X_bf16, M, N, K, Y, out);
+    if (r != DMR_OK) return r;
+    if (!W_bf16) return DMR_ERR_INVALID_ARG;
+    if (!aligned16(W_bf16)) return DMR_ERR_ALIGNMENT;
+    dmr_qformat_t f = {4, 0};
+    if (!workspace || workspace_bytes < dmr_workspace_bytes(DMR_OP_DENSE_LINEAR, M, N, K, f)) return DMR_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
+    if (M == 0) return DMR_OK;
+    RowSel sel = {nullptr, nullptr, 0};
+    return run_dense(reinterpret_cast<const uint16_t *>(X_bf16), M, sel, reinterpret_cast<const uint16_t *>(W_bf16), N,
+                     K, Y, out, (cudaStream_t)stream);
+}
+
+dmr_status_t dmr_route_partition(const uint8_t *mask, int M, int32_t *idx_high, int32_t *idx_low,
+                                 int32_t *counts, void *stream) {
+    if (M < 0 || !counts) return DMR_ERR_INVALID_ARG;
+    if (M > 0 && (!mask || !idx_high || !idx_low)) return DMR_ERR_INVALID_ARG;
+    return launch_route_partition(mask, M, idx_high, idx_low, counts, (cudaStream_t)stream);
+}
+
+dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, const void *W_bf16,
+                               const void *qweight, const void *scales, const void *zeros, int N, int K,
+                               dmr_qformat_t f, void *Y, dmr_out_t out, void *workspace,
+                               size_t workspace_bytes, void *stream) {
+    dmr_status_t r = common_checks(X_bf16, M, N, K, Y, out);
+    if (r != DMR_OK) return r;
+    if (!W_bf16 || !qweight || !scales || !zeros) return DMR_ERR_INVALID_ARG;
+    if (M > 0 && !mask) return DMR_ERR_INVALID_ARG;
+    if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
+    if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
+    if (!aligned16(W_bf16) || !aligned16(qweight)) return DMR_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < dmr_workspace_bytes(DMR_OP_ROUTED_LINEAR, M, N, K, f)) return DMR_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
+    if (M == 0) return DMR_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    RoutedWs w = carve_routed(workspace, M);
+    r = launch_route_partition(mask, M, w.idx_high, w.idx_low, w.counts, st);
+    if (r != DMR_OK) return r;
+    const uint16_t *X = reinterpret_cast<const uint16_t *>(X_bf16);
+    RowSel low = {w.idx_low, w.counts + 1, 0};
+    r = run_lowbit(X, M, low, reinterpret_cast<const uint32_t *>(qweight), reinterpret_cast<const uint16_t *>(scales),
+                   reinterpret_cast<const uint8_t *>(zeros), N, K, f, Y, out, st);
+    if (r != DMR_OK) return r;
+    RowSel high = {w.idx_high, w.counts + 0, 0};
+    return run_dense(X, M, high, reinterpret_cast<const uint16_t *>(W_bf16), N, K, Y, out, st);
+}
+
+size_t dmr_host_staging_bytes(int M, int N, int K, dmr_out_t out) {
+    if (M < 0 || N < 1 || K < 1) return 0;
+    return round_up((size_t)M * K * 2, 256) + round_up((size_t)M * N * (out == DMR_OUT_F32 ? 4 : 2), 256) + 256;
+}
+
+dmr_status_t dmr_lowbit_linear_host(const void *X_host, int M, const void *qweight, const void *scales,
+                                    const void *zeros, int N, int K, dmr_qformat_t f, void *Y_host,
+                                    dmr_out_t out, void *staging, size_t staging_bytes, void *workspace,
+                                    size_t workspace_bytes, void *stream) {
+    if (M < 0 || N < 1 || K < 1) return DMR_ERR_INVALID_ARG;
+    if (M > 0 && (!X_host || !Y_host)) return DMR_ERR_INVALID_ARG;
+    if (!staging || staging_bytes < dmr_host_staging_bytes(M, N, K, out)) return DMR_ERR_WORKSPACE;
+    if (!aligned16(staging)) return DMR_ERR_ALIGNMENT;
+    if (M == 0) return DMR_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t xbytes = (size_t)M * K * 2, ybytes = (size_t)M * N * (out == DMR_OUT_F32 ? 4 : 2);
+    char *Xd = reinterpret_cast<char *>(staging);
+    char *Yd = Xd + round_up(xbytes, 256);
+    cudaError_t e = cudaMemcpyAsync(Xd, X_host, xbytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return DMR_ERR_CUDA;
+    }
+    dmr_status_t r = dmr_lowbit_linear(Xd, M, qweight, scales, zeros, N, K, f, Yd, out, workspace, workspace_bytes, stream);
+    if (r != DMR_OK) return r;
+    e = cudaMemcpyAsync(Y_host, Yd, ybytes, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return DMR_ERR_CUDA;
+    }
+    return DMR_OK;
+}
+
+dmr_status_t dmr_workspace_status(const void *workspace, void *stream) {
+    if (!workspace) return DMR_ERR_INVALID_ARG;
+    int32_t v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, workspace, sizeof v, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return DMR_ERR_CUDA;
+    }
+    return v == 0 ? DMR_OK : (dmr_status_t)v;
+}
+
+const char *dmr_status_string(dmr_status_t s) {
+    switch (s) {
+        case DMR_OK: return "ok";
+        case DMR_ERR_INVALID_ARG: return "invalid argument";
+        case DMR_ERR_UNSUPPORTED: return "unsupported format or shape";
+        case DMR_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case DMR_ERR_WORKSPACE: return "workspace missing or too small";
+        case DMR_ERR_NONFINITE: return "non-finite weight";
+        case DMR_ERR_TIMEOUT: return "bounded wait ran out on the device";
+        case DMR_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+int dmr_last_cuda_error(void) { return g_last_cuda_error; }
+
+uint64_t dmr_launch_count(void) { return g_launches; }
+
+}  // extern "C"

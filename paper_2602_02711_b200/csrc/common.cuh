@@ -1,0 +1,83 @@
+// Shared declarations of the libdmr CUDA sources (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dmr.h"
+
+namespace dmr {
+
+// ---- host-side bookkeeping -------------------------------------------------------------
+extern int g_last_cuda_error;           // last failing cudaError_t (0 if none)
+extern unsigned long long g_launches;   // kernels launched by this library in this process
+
+inline dmr_status_t check_launch() {
+    ++g_launches;
+    cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        (void)cudaGetLastError();
+        return DMR_ERR_CUDA;
+    }
+    return DMR_OK;
+}
+
+inline bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+inline int group_of(int K, dmr_qformat_t f) { return f.group_size == 0 ? K : f.group_size; }
+
+// A format is usable when: bits in {4,8}; K, g multiples of 32; g divides K.
+inline bool format_ok(int K, dmr_qformat_t f) {
+    if (f.bits != 4 && f.bits != 8) return false;
+    if (K <= 0 || K % 32 != 0) return false;
+    int g = group_of(K, f);
+    if (g <= 0 || g % 32 != 0 || K % g != 0) return false;
+    return true;
+}
+
+// Row lists for routed calls: `idx` lists the rows of X/Y to process and `count` (device) says
+// how many entries are valid.  Both null for a plain call over rows 0..M-1.
+struct RowSel {
+    const int32_t *idx;    // already advanced to the first slot of this launch
+    const int32_t *count;  // total number of valid slots in the list
+    int32_t offset;        // list position of this launch's first slot (subtracted from *count)
+};
+
+// ---- workspace layout --------------------------------------------------------------------
+// [0, 256)            status word (int32) + padding
+// [256, ...)          routed: counts[2] (+pad to 256), idx_high[Mpad], idx_low[Mpad]
+// then                compacted activations / split-K partial sums, op dependent
+constexpr size_t kWsStatusBytes = 256;
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- kernel launchers (defined in the .cu files) ------------------------------------------
+dmr_status_t launch_quantize(const uint16_t *W, int N, int K, int bits, int g, uint32_t *qweight,
+                             uint16_t *scales, uint8_t *zeros, int32_t *dev_status,
+                             cudaStream_t st);
+dmr_status_t launch_dequantize(const uint32_t *qweight, const uint16_t *scales, const uint8_t *zeros,
+                               int N, int K, int bits, int g, void *W_out, dmr_out_t out,
+                               cudaStream_t st);
+
+// Decode family (M <= 16): tensor-core GEMV streaming the weights once.
+bool decode_lowbit_supported(int M, int N, int K, int bits, int g);
+dmr_status_t launch_decode_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
+                                  const uint16_t *scales, const uint8_t *zeros, int N, int K,
+                                  int bits, int g, void *Y, dmr_out_t out, cudaStream_t st);
+bool decode_dense_supported(int M, int N, int K);
+dmr_status_t launch_decode_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N,
+                                 int K, void *Y, dmr_out_t out, cudaStream_t st);
+
+// Any-shape fallback (CUDA cores, one warp per output feature).
+dmr_status_t launch_simple_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
+                                  const uint16_t *scales, const uint8_t *zeros, int N, int K,
+                                  int bits, int g, void *Y, dmr_out_t out, cudaStream_t st);
+dmr_status_t launch_simple_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N,
+                                 int K, void *Y, dmr_out_t out, cudaStream_t st);
+
+// Route partition.
+dmr_status_t launch_route_partition(const uint8_t *mask, int M, int32_t *idx_high, int32_t *idx_low,
+                                    int32_t *counts, cudaStream_t st);
+
+}  // namespace dmr

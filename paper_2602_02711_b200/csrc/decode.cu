@@ -1,0 +1,579 @@
+// Decode-time linear layers (M <= 16 rows): bandwidth-bound kernels that stream the weight
+// matrix exactly once.  Decoding re-streams the model weights for every generated token and is
+// limited by memory bandwidth, which is where weight-only quantization pays (App. "Evaluation
+// protocol", discussion of output length; App. "Latency coefficients").
+//
+// Shape of the computation.  A CTA owns 16*R consecutive output features and its 8 warps split K
+// into 8 contiguous slices; partial sums meet in shared memory and are added in warp order, so
+// the summation order of an output depends on (K) only - not on M, on the row's position in the
+// batch or on the other rows.  Inside a warp the product runs on the tensor cores with the
+// weights as the 16-row operand of mma.m16n8k16 (bf16 in, fp32 accumulate) and up to 8 (or
+// 2 x 8) activation rows as the 8-column operand.  Packed codes go from global memory to
+// registers with 128-bit loads, are unpacked with one LOP3 per two codes
+// ((w >> 4p) & 0x000F000F | 0x43004300 = {128+q_p, 128+q_{p+4}} as two bf16) and dequantized with
+// two packed bf16 instructions per pair: (v - (128+zero)) * scale, which is the nearest bf16 of
+// scale*(q-zero).  Which k each fragment slot holds is free as long as both operands agree, so
+// the activation fragments are permuted to the unpack order instead of the weights.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace dmr {
+
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+
+__device__ __forceinline__ uint4 ldg_stream(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint4 ldg_cached(const void *p) {
+    return __ldg(reinterpret_cast<const uint4 *>(p));
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));  // (a & b) | c
+    return r;
+}
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t bf16x2_sub(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// Row of X (and of Y) that batch slot `slot` stands for; -1 if the slot is empty.
+__device__ __forceinline__ int slot_row(int slot, int rows, const int32_t *idx) {
+    if (slot >= rows) return -1;
+    return idx ? idx[slot] : slot;
+}
+
+// Cross-warp reduction in fixed warp order and store of the CTA's [16R features] x [8NT slots].
+template <int NT, int R, bool OUT_F32>
+__device__ __forceinline__ void reduce_and_store(float (&acc)[R][NT][4], float *red, int n0, int N,
+                                                 int rows, const int32_t *idx, void *Y) {
+    constexpr int FEAT = 16 * R, SLOTS = 8 * NT;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    float *mine = red + (size_t)warp * FEAT * SLOTS;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int s0 = nt * 8 + 2 * t;
+            mine[(s0 + 0) * FEAT + r * 16 + g] = acc[r][nt][0];
+            mine[(s0 + 1) * FEAT + r * 16 + g] = acc[r][nt][1];
+            mine[(s0 + 0) * FEAT + r * 16 + g + 8] = acc[r][nt][2];
+            mine[(s0 + 1) * FEAT + r * 16 + g + 8] = acc[r][nt][3];
+        }
+    __syncthreads();
+    for (int o = threadIdx.x; o < FEAT * SLOTS; o += kThreads) {
+        const int slot = o / FEAT, f = o % FEAT;
+        const int row = slot_row(slot, rows, idx);
+        const int n = n0 + f;
+        if (row < 0 || n >= N) continue;
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) s += red[(size_t)w * FEAT * SLOTS + o];
+        if (OUT_F32)
+            reinterpret_cast<float *>(Y)[(size_t)row * N + n] = s;
+        else
+            reinterpret_cast<__nv_bfloat16 *>(Y)[(size_t)row * N + n] = __float2bfloat16_rn(s);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Low-bit weights.  One step = 128 consecutive k; lane (g = lane/4, t = lane%4) owns codes
+// [32t, 32t+32) of the step for features g and g+8 of each 16-feature tile.
+// ---------------------------------------------------------------------------------------------
+template <int BITS, int NT, int R, bool OUT_F32>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_lowbit_kernel(const uint16_t *__restrict__ X, int M, const int32_t *__restrict__ idx,
+                     const int32_t *__restrict__ count, int coff, const uint32_t *__restrict__ qweight,
+                     const uint16_t *__restrict__ scales, const uint8_t *__restrict__ zeros, int N,
+                     int K, int g_size, void *__restrict__ Y) {
+    extern __shared__ float red[];
+    const int rows = count ? min(*count - coff, M) : M;
+    if (rows <= 0) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const int n0 = blockIdx.x * 16 * R;
+    const int G = K / g_size;
+    constexpr int WPR = BITS == 4 ? 4 : 8;  // 32-bit words per lane per feature per step
+
+    const int steps = K / 128;
+    const int spw = (steps + kWarps - 1) / kWarps;
+    const int s_begin = warp * spw, s_end = min(steps, s_begin + spw);
+
+    // feature rows this lane reads (clamped at the matrix edge; edge results are not stored)
+    int frow[R][2];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        frow[r][0] = min(n0 + r * 16 + g, N - 1);
+        frow[r][1] = min(n0 + r * 16 + g + 8, N - 1);
+    }
+    // activation rows of this lane's fragment column
+    int xrow[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) xrow[nt] = slot_row(nt * 8 + g, rows, idx);
+
+    float acc[R][NT][4];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[r][nt][c] = 0.f;
+
+    const size_t words_per_row = (size_t)K * BITS / 32;
+    uint32_t wq[R][2][WPR];
+    auto load_weights = [&](int s) {
+        const size_t woff = ((size_t)s * 128 + 32 * t) * BITS / 32;
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t *p = qweight + (size_t)frow[r][h] * words_per_row + woff;
+#pragma unroll
+                for (int v = 0; v < WPR / 4; ++v) {
+                    uint4 q = ldg_stream(p + 4 * v);
+                    wq[r][h][4 * v + 0] = q.x;
+                    wq[r][h][4 * v + 1] = q.y;
+                    wq[r][h][4 * v + 2] = q.z;
+                    wq[r][h][4 * v + 3] = q.w;
+                }
+            }
+    };
+
+    if (s_begin < s_end) load_weights(s_begin);
+
+    for (int s = s_begin; s < s_end; ++s) {
+        const int kc = s * 128 + 32 * t;  // first k of this lane's chunk
+        const int grp = kc / g_size;
+
+        // activation fragments for this step: x[nt][i] = the two bf16 at k = kc + 2i, kc + 2i + 1
+        uint32_t xb[NT][16];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            if (xrow[nt] >= 0) {
+                const uint16_t *xp = X + (size_t)xrow[nt] * K + kc;
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    uint4 q = ldg_cached(xp + 8 * v);
+                    xb[nt][4 * v + 0] = q.x;
+                    xb[nt][4 * v + 1] = q.y;
+                    xb[nt][4 * v + 2] = q.z;
+                    xb[nt][4 * v + 3] = q.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) xb[nt][i] = 0u;
+            }
+        }
+
+        // scale / zero of (feature, group) for this lane's chunk
+        uint32_t sc2[R][2];
+        uint32_t zc[R][2];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const size_t gi = (size_t)frow[r][h] * G + grp;
+                const uint32_t sb = __ldg(scales + gi);
+                const uint32_t zb = __ldg(zeros + gi);
+                sc2[r][h] = sb | (sb << 16);
+                zc[r][h] = zb;
+            }
+
+        // current weights -> local copy, then prefetch the next step
+        uint32_t cur[R][2][WPR];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int v = 0; v < WPR; ++v) cur[r][h][v] = wq[r][h][v];
+        if (s + 1 < s_end) load_weights(s + 1);
+
+        if (BITS == 4) {
+            // permute activations to the unpack order: pairs (k+p, k+p+4)
+            uint32_t bfrag[NT][8][2];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t r0 = xb[nt][4 * i + 0], r1 = xb[nt][4 * i + 1];
+                    const uint32_t r2 = xb[nt][4 * i + 2], r3 = xb[nt][4 * i + 3];
+                    bfrag[nt][2 * i + 0][0] = prmt(r0, r2, 0x5410);  // (x0, x4)
+                    bfrag[nt][2 * i + 0][1] = prmt(r0, r2, 0x7632);  // (x1, x5)
+                    bfrag[nt][2 * i + 1][0] = prmt(r1, r3, 0x5410);  // (x2, x6)
+                    bfrag[nt][2 * i + 1][1] = prmt(r1, r3, 0x7632);  // (x3, x7)
+                }
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                uint32_t zoff[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t zz = 0x4300u | zc[r][h];  // bf16 of 128 + zero (exact)
+                    zoff[h] = zz | (zz << 16);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int p = 2 * hh;
+                        uint32_t a[4];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t u = cur[r][h][i];
+                            const uint32_t v0 = lop3_and_or(u >> (4 * p), 0x000F000Fu, 0x43004300u);
+                            const uint32_t v1 = lop3_and_or(u >> (4 * p + 4), 0x000F000Fu, 0x43004300u);
+                            a[h] = bf16x2_mul(bf16x2_sub(v0, zoff[h]), sc2[r][h]);      // codes p, p+4
+                            a[2 + h] = bf16x2_mul(bf16x2_sub(v1, zoff[h]), sc2[r][h]);  // codes p+1, p+5
+                        }
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt)
+                            mma_bf16_16816(acc[r][nt], a[0], a[1], a[2], a[3], bfrag[nt][2 * i + hh][0],
+                                           bfrag[nt][2 * i + hh][1]);
+                    }
+                }
+            }
+        } else {
+            // 8-bit codes: byte -> fp32 through the 2^23 mantissa trick, (q - zero) * scale exactly in
+            // fp32, then one rounding to bf16.  Pairs stay in natural k order.
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float sf[2], zf[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    sf[h] = __uint_as_float(sc2[r][h] << 16);
+                    zf[h] = __uint_as_float(0x4B000000u | zc[r][h]);  // 2^23 + zero
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    uint32_t a[4];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t u = cur[r][h][i];
+                        float f[4];
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+                            const uint32_t m = prmt(u, 0x4B000000u, 0x7650u + (uint32_t)b);  // 2^23 + byte b
+                            f[b] = __fmul_rn(__fsub_rn(__uint_as_float(m), zf[h]), sf[h]);
+                        }
+                        a[h] = pack_bf16x2_rn(f[0], f[1]);
+                        a[2 + h] = pack_bf16x2_rn(f[2], f[3]);
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+                        mma_bf16_16816(acc[r][nt], a[0], a[1], a[2], a[3], xb[nt][2 * i], xb[nt][2 * i + 1]);
+                }
+            }
+        }
+    }
+
+    reduce_and_store<NT, R, OUT_F32>(acc, red, n0, N, rows, idx, Y);
+}
+
+// ---------------------------------------------------------------------------------------------
+// bf16 weights (the high-precision rows).  One step = 64 consecutive k; lane (g, t) owns
+// k = 32i + 8t .. +8 (i = 0, 1) of the step for features g and g+8.
+// ---------------------------------------------------------------------------------------------
+template <int NT, int R, bool OUT_F32>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_dense_kernel(const uint16_t *__restrict__ X, int M, const int32_t *__restrict__ idx,
+                    const int32_t *__restrict__ count, int coff, const uint16_t *__restrict__ W, int N, int K,
+                    void *__restrict__ Y) {
+    extern __shared__ float red[];
+    const int rows = count ? min(*count - coff, M) : M;
+    if (rows <= 0) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const int n0 = blockIdx.x * 16 * R;
+
+    const int steps = K / 64;
+    const int spw = (steps + kWarps - 1) / kWarps;
+    const int s_begin = warp * spw, s_end = min(steps, s_begin + spw);
+
+    int frow[R][2];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        frow[r][0] = min(n0 + r * 16 + g, N - 1);
+        frow[r][1] = min(n0 + r * 16 + g + 8, N - 1);
+    }
+    int xrow[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) xrow[nt] = slot_row(nt * 8 + g, rows, idx);
+
+    float acc[R][NT][4];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[r][nt][c] = 0.f;
+
+    uint4 wv[R][2][2];
+    auto load_weights = [&](int s) {
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+                    wv[r][h][i] = ldg_stream(W + (size_t)frow[r][h] * K + (size_t)s * 64 + 32 * i + 8 * t);
+    };
+    if (s_begin < s_end) load_weights(s_begin);
+
+    for (int s = s_begin; s < s_end; ++s) {
+        uint4 xv[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                if (xrow[nt] >= 0)
+                    xv[nt][i] = ldg_cached(X + (size_t)xrow[nt] * K + (size_t)s * 64 + 32 * i + 8 * t);
+                else
+                    xv[nt][i] = make_uint4(0, 0, 0, 0);
+            }
+        uint4 cur[R][2][2];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int i = 0; i < 2; ++i) cur[r][h][i] = wv[r][h][i];
+        if (s + 1 < s_end) load_weights(s + 1);
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    mma_bf16_16816(acc[r][nt], cur[r][0][i].x, cur[r][1][i].x, cur[r][0][i].y,
+                                   cur[r][1][i].y, xv[nt][i].x, xv[nt][i].y);
+                    mma_bf16_16816(acc[r][nt], cur[r][0][i].z, cur[r][1][i].z, cur[r][0][i].w,
+                                   cur[r][1][i].w, xv[nt][i].z, xv[nt][i].w);
+                }
+    }
+    reduce_and_store<NT, R, OUT_F32>(acc, red, n0, N, rows, idx, Y);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Any-shape fallback: one warp per output feature, fp32 FMAs, lanes stride over k in chunks of 8.
+// ---------------------------------------------------------------------------------------------
+template <int MODE /*0 dense, 4, 8*/, bool OUT_F32>
+__global__ void __launch_bounds__(256)
+simple_linear_kernel(const uint16_t *__restrict__ X, int M, const int32_t *__restrict__ idx,
+                     const int32_t *__restrict__ count, int coff, const void *__restrict__ Wany,
+                     const uint16_t *__restrict__ scales, const uint8_t *__restrict__ zeros, int N,
+                     int K, int g_size, void *__restrict__ Y) {
+    const int rows = count ? min(*count - coff, M) : M;
+    const int lane = threadIdx.x & 31;
+    const int n = (int)(((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    if (n >= N) return;
+    const int G = MODE == 0 ? 1 : K / g_size;
+    for (int slot = 0; slot < rows; ++slot) {
+        const int row = idx ? idx[slot] : slot;
+        float acc = 0.f;
+        for (int k0 = lane * 8; k0 < K; k0 += 256) {
+            float w[8];
+            if (MODE == 0) {
+                const uint16_t *wp = reinterpret_cast<const uint16_t *>(Wany) + (size_t)n * K + k0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) w[j] = __uint_as_float((uint32_t)wp[j] << 16);
+            } else {
+                const float s = __uint_as_float((uint32_t)scales[(size_t)n * G + k0 / g_size] << 16);
+                const float z = (float)zeros[(size_t)n * G + k0 / g_size];
+                const uint32_t *qp = reinterpret_cast<const uint32_t *>(Wany);
+                if (MODE == 4) {
+                    const uint32_t u = qp[(size_t)n * (K / 8) + k0 / 8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) w[j] = s * ((float)((u >> (4 * j)) & 0xFu) - z);
+                } else {
+                    const uint32_t u0 = qp[(size_t)n * (K / 4) + k0 / 4], u1 = qp[(size_t)n * (K / 4) + k0 / 4 + 1];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        w[j] = s * ((float)((u0 >> (8 * j)) & 0xFFu) - z);
+                        w[4 + j] = s * ((float)((u1 >> (8 * j)) & 0xFFu) - z);
+                    }
+                }
+            }
+            const uint16_t *xp = X + (size_t)row * K + k0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc = fmaf(__uint_as_float((uint32_t)xp[j] << 16), w[j], acc);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+        if (lane == 0) {
+            if (OUT_F32)
+                reinterpret_cast<float *>(Y)[(size_t)row * N + n] = acc;
+            else
+                reinterpret_cast<__nv_bfloat16 *>(Y)[(size_t)row * N + n] = __float2bfloat16_rn(acc);
+        }
+    }
+}
+
+// Features per CTA: keep at least ~2 CTAs per SM when N allows it.
+int pick_r(int N) {
+    if (N >= 148 * 2 * 64) return 4;
+    if (N >= 148 * 2 * 32) return 2;
+    return 1;
+}
+
+template <typename KernelT>
+dmr_status_t set_smem(KernelT kernel, size_t bytes) {
+    if (bytes > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            return DMR_ERR_CUDA;
+        }
+    }
+    return DMR_OK;
+}
+
+template <int BITS, int NT, int R>
+dmr_status_t launch_lowbit_t(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
+                             const uint16_t *scales, const uint8_t *zeros, int N, int K, int g, void *Y,
+                             dmr_out_t out, cudaStream_t st) {
+    const size_t smem = (size_t)kWarps * 16 * R * 8 * NT * sizeof(float);
+    const int grid = (N + 16 * R - 1) / (16 * R);
+    if (out == DMR_OUT_F32) {
+        auto k = decode_lowbit_kernel<BITS, NT, R, true>;
+        if (set_smem(k, smem) != DMR_OK) return DMR_ERR_CUDA;
+        k<<<grid, kThreads, smem, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+    } else {
+        auto k = decode_lowbit_kernel<BITS, NT, R, false>;
+        if (set_smem(k, smem) != DMR_OK) return DMR_ERR_CUDA;
+        k<<<grid, kThreads, smem, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+    }
+    return check_launch();
+}
+
+template <int BITS, int NT>
+dmr_status_t launch_lowbit_r(int R, const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
+                             const uint16_t *scales, const uint8_t *zeros, int N, int K, int g, void *Y,
+                             dmr_out_t out, cudaStream_t st) {
+    switch (R) {
+        case 4: return launch_lowbit_t<BITS, NT, 4>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+        case 2: return launch_lowbit_t<BITS, NT, 2>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+        default: return launch_lowbit_t<BITS, NT, 1>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+    }
+}
+
+template <int NT, int R>
+dmr_status_t launch_dense_t(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N, int K, void *Y,
+                            dmr_out_t out, cudaStream_t st) {
+    const size_t smem = (size_t)kWarps * 16 * R * 8 * NT * sizeof(float);
+    const int grid = (N + 16 * R - 1) / (16 * R);
+    if (out == DMR_OUT_F32) {
+        auto k = decode_dense_kernel<NT, R, true>;
+        if (set_smem(k, smem) != DMR_OK) return DMR_ERR_CUDA;
+        k<<<grid, kThreads, smem, st>>>(X, M, sel.idx, sel.count, sel.offset, W, N, K, Y);
+    } else {
+        auto k = decode_dense_kernel<NT, R, false>;
+        if (set_smem(k, smem) != DMR_OK) return DMR_ERR_CUDA;
+        k<<<grid, kThreads, smem, st>>>(X, M, sel.idx, sel.count, sel.offset, W, N, K, Y);
+    }
+    return check_launch();
+}
+
+}  // namespace
+
+bool decode_lowbit_supported(int M, int N, int K, int bits, int g) {
+    (void)N;
+    return M >= 1 && M <= 16 && K % 128 == 0 && g % 32 == 0 && (bits == 4 || bits == 8);
+}
+
+dmr_status_t launch_decode_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
+                                  const uint16_t *scales, const uint8_t *zeros, int N, int K, int bits,
+                                  int g, void *Y, dmr_out_t out, cudaStream_t st) {
+    const int R = pick_r(N);
+    if (bits == 4) {
+        if (M <= 8) return launch_lowbit_r<4, 1>(R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+        return launch_lowbit_r<4, 2>(R > 2 ? 2 : R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+    }
+    if (M <= 8) return launch_lowbit_r<8, 1>(R > 2 ? 2 : R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+    return launch_lowbit_r<8, 2>(R > 2 ? 2 : R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+}
+
+bool decode_dense_supported(int M, int N, int K) {
+    (void)N;
+    return M >= 1 && M <= 16 && K % 64 == 0;
+}
+
+dmr_status_t launch_decode_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N, int K,
+                                 void *Y, dmr_out_t out, cudaStream_t st) {
+    const int R = pick_r(N) >= 2 ? 2 : 1;
+    if (M <= 8) {
+        if (R == 2) return launch_dense_t<1, 2>(X, M, sel, W, N, K, Y, out, st);
+        return launch_dense_t<1, 1>(X, M, sel, W, N, K, Y, out, st);
+    }
+    if (R == 2) return launch_dense_t<2, 2>(X, M, sel, W, N, K, Y, out, st);
+    return launch_dense_t<2, 1>(X, M, sel, W, N, K, Y, out, st);
+}
+
+dmr_status_t launch_simple_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
+                                  const uint16_t *scales, const uint8_t *zeros, int N, int K, int bits,
+                                  int g, void *Y, dmr_out_t out, cudaStream_t st) {
+    const int grid = (N + 7) / 8;
+    if (bits == 4) {
+        if (out == DMR_OUT_F32)
+            simple_linear_kernel<4, true><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+        else
+            simple_linear_kernel<4, false><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+    } else {
+        if (out == DMR_OUT_F32)
+            simple_linear_kernel<8, true><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+        else
+            simple_linear_kernel<8, false><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+    }
+    return check_launch();
+}
+
+dmr_status_t launch_simple_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N, int K,
+                                 void *Y, dmr_out_t out, cudaStream_t st) {
+    const int grid = (N + 7) / 8;
+    if (out == DMR_OUT_F32)
+        simple_linear_kernel<0, true><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, W, nullptr, nullptr, N, K, K, Y);
+    else
+        simple_linear_kernel<0, false><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, W, nullptr, nullptr, N, K, K, Y);
+    return check_launch();
+}
+
+}  // namespace dmr
