@@ -11,24 +11,57 @@ unsigned long long g_launches = 0;
 
 namespace {
 
-struct RoutedWs {
-    int32_t *counts;    // {n_high, n_low}
-    int32_t *idx_high;  // [Mpad]
-    int32_t *idx_low;   // [Mpad]
-    size_t end;         // bytes used from the workspace base
+// Workspace layout (all offsets multiples of 256 bytes):
+//   [0, 256)   status word
+//   routed:    counts {n_high, n_low} (256 B), idx_high [M], idx_low [M]
+//   routed, tensor-core path: gathered activations of the low rows [M][K], then of the high rows
+//   split-K:   fp32 partial sums [splits][M][N] (shared by the two halves of a routed call)
+struct Scratch {
+    int32_t *status = nullptr;
+    int32_t *counts = nullptr, *idx_high = nullptr, *idx_low = nullptr;
+    uint16_t *xg_low = nullptr, *xg_high = nullptr;
+    float *partial = nullptr;
+    size_t bytes = 0;
 };
 
-size_t routed_lists_bytes(int M) { return 256 + 2 * round_up((size_t)(M > 0 ? M : 1) * 4, 256); }
+bool use_gemm(int M, int N, int K, int bits, int g) { return gemm_supported(M, N, K, bits, g); }
 
-RoutedWs carve_routed(void *workspace, int M) {
-    char *base = reinterpret_cast<char *>(workspace) + kWsStatusBytes;
-    const size_t list = round_up((size_t)(M > 0 ? M : 1) * 4, 256);
-    RoutedWs w;
-    w.counts = reinterpret_cast<int32_t *>(base);
-    w.idx_high = reinterpret_cast<int32_t *>(base + 256);
-    w.idx_low = reinterpret_cast<int32_t *>(base + 256 + list);
-    w.end = kWsStatusBytes + 256 + 2 * list;
-    return w;
+Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f) {
+    Scratch s;
+    char *base = reinterpret_cast<char *>(workspace);
+    size_t off = kWsStatusBytes;
+    s.status = reinterpret_cast<int32_t *>(base);
+    const int g = format_ok(K, f) ? group_of(K, f) : K;
+    const bool low_gemm = op != DMR_OP_DENSE_LINEAR && use_gemm(M, N, K, f.bits, g);
+    const bool dense_gemm = op != DMR_OP_LOWBIT_LINEAR && use_gemm(M, N, K, 0, K);
+    if (op == DMR_OP_ROUTED_LINEAR) {
+        const size_t list = round_up((size_t)(M > 0 ? M : 1) * 4, 256);
+        s.counts = reinterpret_cast<int32_t *>(base + off);
+        s.idx_high = reinterpret_cast<int32_t *>(base + off + 256);
+        s.idx_low = reinterpret_cast<int32_t *>(base + off + 256 + list);
+        off += 256 + 2 * list;
+        const size_t xg = round_up((size_t)M * K * 2, 256);
+        if (low_gemm) {
+            s.xg_low = reinterpret_cast<uint16_t *>(base + off);
+            off += xg;
+        }
+        if (dense_gemm) {
+            s.xg_high = reinterpret_cast<uint16_t *>(base + off);
+            off += xg;
+        }
+    }
+    size_t partial = 0;
+    if (low_gemm) partial = gemm_plan(M, N, K, f.bits).partial_bytes;
+    if (dense_gemm) {
+        const size_t p2 = gemm_plan(M, N, K, 0).partial_bytes;
+        if (p2 > partial) partial = p2;
+    }
+    if (partial) {
+        s.partial = reinterpret_cast<float *>(base + off);
+        off += round_up(partial, 256);
+    }
+    s.bytes = round_up(off, 256);
+    return s;
 }
 
 dmr_status_t common_checks(const void *X, int M, int N, int K, const void *Y, dmr_out_t out) {
@@ -44,9 +77,18 @@ dmr_status_t common_checks(const void *X, int M, int N, int K, const void *Y, dm
 // from (M, N, K, format) only, never from how many rows a routed call found.
 dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales,
                         const uint8_t *zeros, int N, int K, dmr_qformat_t f, void *Y, dmr_out_t out,
-                        cudaStream_t st) {
+                        const Scratch &ws, cudaStream_t st) {
     const int g = group_of(K, f);
     const size_t ysz = out == DMR_OUT_F32 ? 4 : 2;
+    if (use_gemm(M, N, K, f.bits, g)) {
+        const uint16_t *Xin = X;
+        if (sel.idx) {
+            dmr_status_t r = launch_gather_rows(X, K, M, sel.idx, sel.count, ws.xg_low, st);
+            if (r != DMR_OK) return r;
+            Xin = ws.xg_low;
+        }
+        return launch_gemm(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.partial, ws.status, st);
+    }
     if (!decode_lowbit_supported(M < 16 ? M : 16, N, K, f.bits, g))
         return launch_simple_lowbit(X, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, st);
     for (int m0 = 0; m0 < M; m0 += 16) {
@@ -61,15 +103,24 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
             Xc = X + (size_t)m0 * K;
             Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
         }
-        dmr_status_t r = launch_decode_lowbit(Xc, mc, s, qweight, scales, zeros, N, K, f.bits, g, Yc, out, st);
+        dmr_status_t r = launch_decode_lowbit(Xc, mc, s, qweight, scales, zeros, N, K, f.bits, g, Yc, out, ws.status, st);
         if (r != DMR_OK) return r;
     }
     return DMR_OK;
 }
 
 dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N, int K, void *Y,
-                       dmr_out_t out, cudaStream_t st) {
+                       dmr_out_t out, const Scratch &ws, cudaStream_t st) {
     const size_t ysz = out == DMR_OUT_F32 ? 4 : 2;
+    if (use_gemm(M, N, K, 0, K)) {
+        const uint16_t *Xin = X;
+        if (sel.idx) {
+            dmr_status_t r = launch_gather_rows(X, K, M, sel.idx, sel.count, ws.xg_high, st);
+            if (r != DMR_OK) return r;
+            Xin = ws.xg_high;
+        }
+        return launch_gemm(Xin, M, sel, W, nullptr, nullptr, N, K, 0, K, Y, out, ws.partial, ws.status, st);
+    }
     if (!decode_dense_supported(M < 16 ? M : 16, N, K)) return launch_simple_dense(X, M, sel, W, N, K, Y, out, st);
     for (int m0 = 0; m0 < M; m0 += 16) {
         const int mc = M - m0 < 16 ? M - m0 : 16;
@@ -112,12 +163,8 @@ size_t dmr_zeros_bytes(int N, int K, dmr_qformat_t f) {
 }
 
 size_t dmr_workspace_bytes(dmr_op_t op, int M, int N, int K, dmr_qformat_t f) {
-    (void)N;
-    (void)K;
-    (void)f;
-    size_t b = kWsStatusBytes;
-    if (op == DMR_OP_ROUTED_LINEAR) b += routed_lists_bytes(M);
-    return round_up(b, 256);
+    if (M < 0 || N < 1 || K < 1) return kWsStatusBytes;
+    return carve(nullptr, op, M, N, K, f).bytes;
 }
 
 dmr_status_t dmr_quantize(const void *W_bf16, int N, int K, dmr_qformat_t f, void *qweight, void *scales,
@@ -156,9 +203,10 @@ dmr_status_t dmr_lowbit_linear(const void *X_bf16, int M, const void *qweight, c
     if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
     if (M == 0) return DMR_OK;
     RowSel sel = {nullptr, nullptr, 0};
+    const Scratch ws = carve(workspace, DMR_OP_LOWBIT_LINEAR, M, N, K, f);
     return run_lowbit(reinterpret_cast<const uint16_t *>(X_bf16), M, sel, reinterpret_cast<const uint32_t *>(qweight),
                       reinterpret_cast<const uint16_t *>(scales), reinterpret_cast<const uint8_t *>(zeros), N, K, f,
-                      Y, out, (cudaStream_t)stream);
+                      Y, out, ws, (cudaStream_t)stream);
 }
 
 dmr_status_t dmr_dense_linear(const void *X_bf16, int M, const void *W_bf16, int N, int K, void *Y,
@@ -172,8 +220,9 @@ dmr_status_t dmr_dense_linear(const void *X_bf16, int M, const void *W_bf16, int
     if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
     if (M == 0) return DMR_OK;
     RowSel sel = {nullptr, nullptr, 0};
+    const Scratch ws = carve(workspace, DMR_OP_DENSE_LINEAR, M, N, K, f);
     return run_dense(reinterpret_cast<const uint16_t *>(X_bf16), M, sel, reinterpret_cast<const uint16_t *>(W_bf16), N,
-                     K, Y, out, (cudaStream_t)stream);
+                     K, Y, out, ws, (cudaStream_t)stream);
 }
 
 dmr_status_t dmr_route_partition(const uint8_t *mask, int M, int32_t *idx_high, int32_t *idx_low,
@@ -198,16 +247,16 @@ dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, c
     if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
     if (M == 0) return DMR_OK;
     cudaStream_t st = (cudaStream_t)stream;
-    RoutedWs w = carve_routed(workspace, M);
-    r = launch_route_partition(mask, M, w.idx_high, w.idx_low, w.counts, st);
+    const Scratch ws = carve(workspace, DMR_OP_ROUTED_LINEAR, M, N, K, f);
+    r = launch_route_partition(mask, M, ws.idx_high, ws.idx_low, ws.counts, st);
     if (r != DMR_OK) return r;
     const uint16_t *X = reinterpret_cast<const uint16_t *>(X_bf16);
-    RowSel low = {w.idx_low, w.counts + 1, 0};
+    RowSel low = {ws.idx_low, ws.counts + 1, 0};
     r = run_lowbit(X, M, low, reinterpret_cast<const uint32_t *>(qweight), reinterpret_cast<const uint16_t *>(scales),
-                   reinterpret_cast<const uint8_t *>(zeros), N, K, f, Y, out, st);
+                   reinterpret_cast<const uint8_t *>(zeros), N, K, f, Y, out, ws, st);
     if (r != DMR_OK) return r;
-    RowSel high = {w.idx_high, w.counts + 0, 0};
-    return run_dense(X, M, high, reinterpret_cast<const uint16_t *>(W_bf16), N, K, Y, out, st);
+    RowSel high = {ws.idx_high, ws.counts + 0, 0};
+    return run_dense(X, M, high, reinterpret_cast<const uint16_t *>(W_bf16), N, K, Y, out, ws, st);
 }
 
 size_t dmr_host_staging_bytes(int M, int N, int K, dmr_out_t out) {

@@ -64,10 +64,28 @@ dmr_status_t launch_dequantize(const uint32_t *qweight, const uint16_t *scales, 
 bool decode_lowbit_supported(int M, int N, int K, int bits, int g);
 dmr_status_t launch_decode_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
                                   const uint16_t *scales, const uint8_t *zeros, int N, int K,
-                                  int bits, int g, void *Y, dmr_out_t out, cudaStream_t st);
+                                  int bits, int g, void *Y, dmr_out_t out, int32_t *status,
+                                  cudaStream_t st);
 bool decode_dense_supported(int M, int N, int K);
 dmr_status_t launch_decode_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N,
                                  int K, void *Y, dmr_out_t out, cudaStream_t st);
+
+// Tensor-core GEMM family (M > 16): tcgen05 MMA with TMA-staged operands.
+struct GemmPlan {
+    int bn;                 // activation rows per CTA (MMA N)
+    int splits;             // split-K factor (partials are added in split order)
+    int kblocks_per_split;  // 64-wide k blocks per split
+    size_t partial_bytes;   // fp32 partial-sum scratch needed (0 when splits == 1)
+};
+bool gemm_supported(int M, int N, int K, int bits /*0 = bf16 weights*/, int g);
+GemmPlan gemm_plan(int M, int N, int K, int bits);
+// `weights` is W (bits == 0) or qweight.  X holds M rows (for a routed call: the gathered rows,
+// sel.count of them valid); sel.idx maps batch slots to output rows.
+dmr_status_t launch_gemm(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,
+                         const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
+                         float *partial, int32_t *status, cudaStream_t st);
+dmr_status_t launch_gather_rows(const uint16_t *X, int K, int Mcap, const int32_t *idx, const int32_t *count,
+                                uint16_t *Xg, cudaStream_t st);
 
 // Any-shape fallback (CUDA cores, one warp per output feature).
 dmr_status_t launch_simple_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,

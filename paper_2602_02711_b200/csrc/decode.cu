@@ -8,15 +8,21 @@
 // the summation order of an output depends on (K) only - not on M, on the row's position in the
 // batch or on the other rows.  Inside a warp the product runs on the tensor cores with the
 // weights as the 16-row operand of mma.m16n8k16 (bf16 in, fp32 accumulate) and up to 8 (or
-// 2 x 8) activation rows as the 8-column operand.  Packed codes go from global memory to
-// registers with 128-bit loads, are unpacked with one LOP3 per two codes
-// ((w >> 4p) & 0x000F000F | 0x43004300 = {128+q_p, 128+q_{p+4}} as two bf16) and dequantized with
-// two packed bf16 instructions per pair: (v - (128+zero)) * scale, which is the nearest bf16 of
-// scale*(q-zero).  Which k each fragment slot holds is free as long as both operands agree, so
-// the activation fragments are permuted to the unpack order instead of the weights.
+// 2 x 8) activation rows as the 8-column operand.
+//
+// Low-bit weights: every warp runs its own TMA pipeline (cp.async.bulk.tensor into a private ring
+// of 128-byte-swizzled [16R rows x 128 bytes] boxes, one mbarrier per stage), so many kilobytes
+// per SM are in flight without costing registers.  Codes are unpacked with one LOP3 per two codes
+// ((w >> 4p) & 0x000F000F | 0x43004300 = {128+q_p, 128+q_{p+4}} as two bf16) and one packed
+// subtract of (128 + zero): the tensor-core operand is the exact integer q - zero.  Products are
+// accumulated per quantization group in fp32 and the group's scale is applied to the group sum,
+// so no weight is ever rounded: the only error against exact arithmetic is fp32 summation.
+// Which k each fragment slot holds is free as long as both operands agree, so the activation
+// fragments are permuted to the unpack order instead of the weights; which feature each fragment
+// row holds is free too, which is used to make the shared-memory reads conflict-free.
 #include <cuda_bf16.h>
 
-#include "common.cuh"
+#include "sm100.cuh"
 
 namespace dmr {
 
@@ -82,23 +88,34 @@ __device__ __forceinline__ int slot_row(int slot, int rows, const int32_t *idx) 
     return idx ? idx[slot] : slot;
 }
 
+// Fragment row g of a 16-row tile holds tile row tile_row_of(g) (and that + 8).
+template <int BITS>
+__device__ __forceinline__ int tile_row_of(int g) {
+    // 4-bit: rows 0,4,1,5,... so that the eight lanes of one shared-memory phase (two values of g)
+    // land on different 16-byte columns under the 128-byte swizzle.  Otherwise identity.
+    return BITS == 4 ? ((g >> 1) | ((g & 1) << 2)) : g;
+}
+
 // Cross-warp reduction in fixed warp order and store of the CTA's [16R features] x [8NT slots].
-template <int NT, int R, bool OUT_F32>
+// Warp w parks its partial sums at red + w * WSTRIDE floats.
+template <int BITS, int NT, int R, int WSTRIDE, bool OUT_F32>
 __device__ __forceinline__ void reduce_and_store(float (&acc)[R][NT][4], float *red, int n0, int N,
                                                  int rows, const int32_t *idx, void *Y) {
     constexpr int FEAT = 16 * R, SLOTS = 8 * NT;
+    static_assert(WSTRIDE >= FEAT * SLOTS, "partial-sum area too small");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
-    float *mine = red + (size_t)warp * FEAT * SLOTS;
+    const int trow = tile_row_of<BITS>(g);
+    float *mine = red + (size_t)warp * WSTRIDE;
 #pragma unroll
     for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             const int s0 = nt * 8 + 2 * t;
-            mine[(s0 + 0) * FEAT + r * 16 + g] = acc[r][nt][0];
-            mine[(s0 + 1) * FEAT + r * 16 + g] = acc[r][nt][1];
-            mine[(s0 + 0) * FEAT + r * 16 + g + 8] = acc[r][nt][2];
-            mine[(s0 + 1) * FEAT + r * 16 + g + 8] = acc[r][nt][3];
+            mine[(s0 + 0) * FEAT + r * 16 + trow] = acc[r][nt][0];
+            mine[(s0 + 1) * FEAT + r * 16 + trow] = acc[r][nt][1];
+            mine[(s0 + 0) * FEAT + r * 16 + trow + 8] = acc[r][nt][2];
+            mine[(s0 + 1) * FEAT + r * 16 + trow + 8] = acc[r][nt][3];
         }
     __syncthreads();
     for (int o = threadIdx.x; o < FEAT * SLOTS; o += kThreads) {
@@ -108,7 +125,7 @@ __device__ __forceinline__ void reduce_and_store(float (&acc)[R][NT][4], float *
         if (row < 0 || n >= N) continue;
         float s = 0.f;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) s += red[(size_t)w * FEAT * SLOTS + o];
+        for (int w = 0; w < kWarps; ++w) s += red[(size_t)w * WSTRIDE + o];
         if (OUT_F32)
             reinterpret_cast<float *>(Y)[(size_t)row * N + n] = s;
         else
@@ -117,196 +134,222 @@ __device__ __forceinline__ void reduce_and_store(float (&acc)[R][NT][4], float *
 }
 
 // ---------------------------------------------------------------------------------------------
-// Low-bit weights.  One step = 128 consecutive k; lane (g = lane/4, t = lane%4) owns codes
-// [32t, 32t+32) of the step for features g and g+8 of each 16-feature tile.
+// Low-bit weights.  One step of a warp = one TMA box = 128 bytes of each of 16R feature rows
+// (256 4-bit codes or 128 8-bit codes).  A step is consumed in units of UNIT = 128 or 64
+// consecutive k (one quantization group, or a part of one); in a unit, lane (g = lane/4,
+// t = lane%4) owns codes [t*UNIT/4, (t+1)*UNIT/4) of two feature rows per 16-row tile.
 // ---------------------------------------------------------------------------------------------
-template <int BITS, int NT, int R, bool OUT_F32>
+template <int BITS, int NT, int R, int UNIT, int D, bool OUT_F32>
 __global__ void __launch_bounds__(kThreads, 1)
-decode_lowbit_kernel(const uint16_t *__restrict__ X, int M, const int32_t *__restrict__ idx,
-                     const int32_t *__restrict__ count, int coff, const uint32_t *__restrict__ qweight,
-                     const uint16_t *__restrict__ scales, const uint8_t *__restrict__ zeros, int N,
-                     int K, int g_size, void *__restrict__ Y) {
-    extern __shared__ float red[];
+decode_lowbit_kernel(const __grid_constant__ CUtensorMap wmap, const uint16_t *__restrict__ X, int M,
+                     const int32_t *__restrict__ idx, const int32_t *__restrict__ count, int coff,
+                     const uint16_t *__restrict__ scales, const uint8_t *__restrict__ zeros, int N, int K,
+                     int g_size, void *__restrict__ Y, int32_t *__restrict__ status) {
+    constexpr int STEP_K = 128 * 8 / BITS;       // codes per 128-byte row
+    constexpr int UNITS = STEP_K / UNIT;         // units per step
+    constexpr int CPL = UNIT / 4;                // codes per lane per unit
+    constexpr int BPL = CPL * BITS / 8;          // bytes per lane per unit (8, 16 or 32)
+    constexpr int WPL = BPL / 4;                 // 32-bit words per lane per unit
+    constexpr int XV = CPL / 8;                  // 16-byte activation loads per lane per unit
+    constexpr int ROWS = 16 * R;
+    constexpr int STAGE_BYTES = ROWS * 128;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+
     const int rows = count ? min(*count - coff, M) : M;
     if (rows <= 0) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
-    const int n0 = blockIdx.x * 16 * R;
+    const int n0 = blockIdx.x * ROWS;
     const int G = K / g_size;
-    constexpr int WPR = BITS == 4 ? 4 : 8;  // 32-bit words per lane per feature per step
 
-    const int steps = K / 128;
+    uint8_t *my_stages = smem_raw + (size_t)warp * D * STAGE_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_raw + (size_t)kWarps * D * STAGE_BYTES) + warp * D;
+    const uint32_t stage0 = smem_u32(my_stages);
+    const uint32_t bar0 = smem_u32(bars);
+
+    const int steps = (K + STEP_K - 1) / STEP_K;
     const int spw = (steps + kWarps - 1) / kWarps;
-    const int s_begin = warp * spw, s_end = min(steps, s_begin + spw);
+    const int s_begin = warp * spw;
+    const int my_steps = max(0, min(steps, s_begin + spw) - s_begin);
 
-    // feature rows this lane reads (clamped at the matrix edge; edge results are not stored)
-    int frow[R][2];
+    if (lane == 0) {
+        for (int d = 0; d < D; ++d) mbar_init(bar0 + 8 * d, 1);
+        fence_barrier_init();
+        for (int d = 0; d < D && d < my_steps; ++d) {
+            mbar_expect_tx(bar0 + 8 * d, STAGE_BYTES);
+            tma_load_2d(stage0 + d * STAGE_BYTES, &wmap, bar0 + 8 * d, (s_begin + d) * 128, n0);
+        }
+    }
+    __syncwarp();
+
+    // tile rows / features of this lane, activation rows of this lane's fragment column
+    const int trow = tile_row_of<BITS>(g);
+    int feat[R][2];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        frow[r][0] = min(n0 + r * 16 + g, N - 1);
-        frow[r][1] = min(n0 + r * 16 + g + 8, N - 1);
+        feat[r][0] = min(n0 + r * 16 + trow, N - 1);
+        feat[r][1] = min(n0 + r * 16 + trow + 8, N - 1);
     }
-    // activation rows of this lane's fragment column
     int xrow[NT];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) xrow[nt] = slot_row(nt * 8 + g, rows, idx);
 
-    float acc[R][NT][4];
+    float acc[R][NT][4], accg[R][NT][4];
 #pragma unroll
     for (int r = 0; r < R; ++r)
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) acc[r][nt][c] = 0.f;
+            for (int c = 0; c < 4; ++c) acc[r][nt][c] = accg[r][nt][c] = 0.f;
 
-    const size_t words_per_row = (size_t)K * BITS / 32;
-    uint32_t wq[R][2][WPR];
-    auto load_weights = [&](int s) {
-        const size_t woff = ((size_t)s * 128 + 32 * t) * BITS / 32;
+    // byte offset of this lane inside a 128-byte row for unit u, before swizzling
+    const uint32_t lane_row_off[2] = {(uint32_t)(trow * 128), (uint32_t)((trow + 8) * 128)};
+    const uint32_t swz = (uint32_t)(trow & 7);  // (trow + 8) & 7 is the same
+
+    bool ok = true;
+    for (int i = 0; i < my_steps && ok; ++i) {
+        const int d = i % D;
+        ok = mbar_wait(bar0 + 8 * d, (uint32_t)((i / D) & 1), status);
+        if (!ok) break;
+        const uint32_t st = stage0 + d * STAGE_BYTES;
+        const int kstep = (s_begin + i) * STEP_K;
 #pragma unroll
-        for (int r = 0; r < R; ++r)
+        for (int u = 0; u < UNITS; ++u) {
+            const int k0 = kstep + u * UNIT;
+            if (k0 >= K) break;  // warp-uniform: the box reached past the end of the row
+            const int grp = k0 / g_size;
+
+            // activations: the two bf16 at k = kc + 2j, kc + 2j + 1 in xb[nt][j]
+            const int kc = k0 + t * CPL;
+            uint32_t xb[NT][4 * XV];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint32_t *p = qweight + (size_t)frow[r][h] * words_per_row + woff;
+            for (int nt = 0; nt < NT; ++nt) {
+                if (xrow[nt] >= 0) {
+                    const uint16_t *xp = X + (size_t)xrow[nt] * K + kc;
 #pragma unroll
-                for (int v = 0; v < WPR / 4; ++v) {
-                    uint4 q = ldg_stream(p + 4 * v);
-                    wq[r][h][4 * v + 0] = q.x;
-                    wq[r][h][4 * v + 1] = q.y;
-                    wq[r][h][4 * v + 2] = q.z;
-                    wq[r][h][4 * v + 3] = q.w;
+                    for (int v = 0; v < XV; ++v) {
+                        uint4 q = ldg_cached(xp + 8 * v);
+                        xb[nt][4 * v + 0] = q.x;
+                        xb[nt][4 * v + 1] = q.y;
+                        xb[nt][4 * v + 2] = q.z;
+                        xb[nt][4 * v + 3] = q.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4 * XV; ++j) xb[nt][j] = 0u;
                 }
             }
-    };
+            // zero points of (feature, group)
+            uint32_t zb[R][2];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) zb[r][h] = __ldg(zeros + (size_t)feat[r][h] * G + grp);
 
-    if (s_begin < s_end) load_weights(s_begin);
-
-    for (int s = s_begin; s < s_end; ++s) {
-        const int kc = s * 128 + 32 * t;  // first k of this lane's chunk
-        const int grp = kc / g_size;
-
-        // activation fragments for this step: x[nt][i] = the two bf16 at k = kc + 2i, kc + 2i + 1
-        uint32_t xb[NT][16];
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            if (xrow[nt] >= 0) {
-                const uint16_t *xp = X + (size_t)xrow[nt] * K + kc;
-#pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    uint4 q = ldg_cached(xp + 8 * v);
-                    xb[nt][4 * v + 0] = q.x;
-                    xb[nt][4 * v + 1] = q.y;
-                    xb[nt][4 * v + 2] = q.z;
-                    xb[nt][4 * v + 3] = q.w;
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) xb[nt][i] = 0u;
-            }
-        }
-
-        // scale / zero of (feature, group) for this lane's chunk
-        uint32_t sc2[R][2];
-        uint32_t zc[R][2];
-#pragma unroll
-        for (int r = 0; r < R; ++r)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const size_t gi = (size_t)frow[r][h] * G + grp;
-                const uint32_t sb = __ldg(scales + gi);
-                const uint32_t zb = __ldg(zeros + gi);
-                sc2[r][h] = sb | (sb << 16);
-                zc[r][h] = zb;
-            }
-
-        // current weights -> local copy, then prefetch the next step
-        uint32_t cur[R][2][WPR];
-#pragma unroll
-        for (int r = 0; r < R; ++r)
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int v = 0; v < WPR; ++v) cur[r][h][v] = wq[r][h][v];
-        if (s + 1 < s_end) load_weights(s + 1);
-
-        if (BITS == 4) {
-            // permute activations to the unpack order: pairs (k+p, k+p+4)
-            uint32_t bfrag[NT][8][2];
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t r0 = xb[nt][4 * i + 0], r1 = xb[nt][4 * i + 1];
-                    const uint32_t r2 = xb[nt][4 * i + 2], r3 = xb[nt][4 * i + 3];
-                    bfrag[nt][2 * i + 0][0] = prmt(r0, r2, 0x5410);  // (x0, x4)
-                    bfrag[nt][2 * i + 0][1] = prmt(r0, r2, 0x7632);  // (x1, x5)
-                    bfrag[nt][2 * i + 1][0] = prmt(r1, r3, 0x5410);  // (x2, x6)
-                    bfrag[nt][2 * i + 1][1] = prmt(r1, r3, 0x7632);  // (x3, x7)
-                }
+            const uint32_t boff = (uint32_t)(u * (UNIT * BITS / 8) + t * BPL);  // logical byte in the row
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                uint32_t zoff[2];
+                // packed codes of this lane: rows trow and trow + 8 of tile r
+                uint32_t wq[2][WPL];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const uint32_t zz = 0x4300u | zc[r][h];  // bf16 of 128 + zero (exact)
-                    zoff[h] = zz | (zz << 16);
+                    const uint32_t rowbase = st + r * 2048 + lane_row_off[h];
+#pragma unroll
+                    for (int c = 0; c < (BPL + 15) / 16; ++c) {
+                        const uint32_t chunk = ((boff >> 4) + c) ^ swz;
+                        const uint32_t addr = rowbase + (chunk << 4) + (boff & 15u);
+                        if (BPL >= 16) {
+                            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                         : "=r"(wq[h][4 * c + 0]), "=r"(wq[h][4 * c + 1]), "=r"(wq[h][4 * c + 2]),
+                                           "=r"(wq[h][4 * c + 3])
+                                         : "r"(addr));
+                        } else {
+                            asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(wq[h][0]), "=r"(wq[h][1]) : "r"(addr));
+                        }
+                    }
                 }
+                if (BITS == 4) {
+                    uint32_t zoff[2];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t zz = 0x4300u | zb[r][h];  // bf16 of 128 + zero (exact)
+                        zoff[h] = zz | (zz << 16);
+                    }
 #pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        const int p = 2 * hh;
+                    for (int w = 0; w < WPL; ++w) {
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            uint32_t a[4];
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const uint32_t uu = wq[h][w];
+                                const uint32_t v0 = lop3_and_or(uu >> (8 * hh), 0x000F000Fu, 0x43004300u);
+                                const uint32_t v1 = lop3_and_or(uu >> (8 * hh + 4), 0x000F000Fu, 0x43004300u);
+                                a[h] = bf16x2_sub(v0, zoff[h]);      // codes p, p+4 (p = 2hh) minus zero
+                                a[2 + h] = bf16x2_sub(v1, zoff[h]);  // codes p+1, p+5
+                            }
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                // activations in the same order: (x_p, x_{p+4}) and (x_{p+1}, x_{p+5})
+                                const uint32_t r0 = xb[nt][4 * w + hh], r2 = xb[nt][4 * w + 2 + hh];
+                                mma_bf16_16816(accg[r][nt], a[0], a[1], a[2], a[3], prmt(r0, r2, 0x5410),
+                                               prmt(r0, r2, 0x7632));
+                            }
+                        }
+                    }
+                } else {
+                    float zf[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) zf[h] = __uint_as_float(0x4B000000u | zb[r][h]);  // 2^23 + zero
+#pragma unroll
+                    for (int w = 0; w < WPL; ++w) {
                         uint32_t a[4];
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const uint32_t u = cur[r][h][i];
-                            const uint32_t v0 = lop3_and_or(u >> (4 * p), 0x000F000Fu, 0x43004300u);
-                            const uint32_t v1 = lop3_and_or(u >> (4 * p + 4), 0x000F000Fu, 0x43004300u);
-                            a[h] = bf16x2_mul(bf16x2_sub(v0, zoff[h]), sc2[r][h]);      // codes p, p+4
-                            a[2 + h] = bf16x2_mul(bf16x2_sub(v1, zoff[h]), sc2[r][h]);  // codes p+1, p+5
+                            const uint32_t uu = wq[h][w];
+                            float f[4];
+#pragma unroll
+                            for (int b = 0; b < 4; ++b)  // (2^23 + byte) - (2^23 + zero) = q - zero exactly
+                                f[b] = __fsub_rn(__uint_as_float(prmt(uu, 0x4B000000u, 0x7650u + (uint32_t)b)), zf[h]);
+                            a[h] = pack_bf16x2_rn(f[0], f[1]);  // |q - zero| <= 255: exact in bf16
+                            a[2 + h] = pack_bf16x2_rn(f[2], f[3]);
                         }
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt)
-                            mma_bf16_16816(acc[r][nt], a[0], a[1], a[2], a[3], bfrag[nt][2 * i + hh][0],
-                                           bfrag[nt][2 * i + hh][1]);
+                            mma_bf16_16816(accg[r][nt], a[0], a[1], a[2], a[3], xb[nt][2 * w], xb[nt][2 * w + 1]);
                     }
                 }
             }
-        } else {
-            // 8-bit codes: byte -> fp32 through the 2^23 mantissa trick, (q - zero) * scale exactly in
-            // fp32, then one rounding to bf16.  Pairs stay in natural k order.
+            // end of a quantization group (or of this warp's slice): apply the group's scale
+            const bool last_unit = (i == my_steps - 1) && (u == UNITS - 1 || k0 + UNIT >= K);
+            if (((k0 + UNIT) % g_size) == 0 || last_unit) {
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                float sf[2], zf[2];
+                for (int r = 0; r < R; ++r) {
+                    const float s0 = __uint_as_float((uint32_t)__ldg(scales + (size_t)feat[r][0] * G + grp) << 16);
+                    const float s1 = __uint_as_float((uint32_t)__ldg(scales + (size_t)feat[r][1] * G + grp) << 16);
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    sf[h] = __uint_as_float(sc2[r][h] << 16);
-                    zf[h] = __uint_as_float(0x4B000000u | zc[r][h]);  // 2^23 + zero
-                }
+                    for (int nt = 0; nt < NT; ++nt) {
+                        acc[r][nt][0] = fmaf(s0, accg[r][nt][0], acc[r][nt][0]);
+                        acc[r][nt][1] = fmaf(s0, accg[r][nt][1], acc[r][nt][1]);
+                        acc[r][nt][2] = fmaf(s1, accg[r][nt][2], acc[r][nt][2]);
+                        acc[r][nt][3] = fmaf(s1, accg[r][nt][3], acc[r][nt][3]);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    uint32_t a[4];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint32_t u = cur[r][h][i];
-                        float f[4];
-#pragma unroll
-                        for (int b = 0; b < 4; ++b) {
-                            const uint32_t m = prmt(u, 0x4B000000u, 0x7650u + (uint32_t)b);  // 2^23 + byte b
-                            f[b] = __fmul_rn(__fsub_rn(__uint_as_float(m), zf[h]), sf[h]);
-                        }
-                        a[h] = pack_bf16x2_rn(f[0], f[1]);
-                        a[2 + h] = pack_bf16x2_rn(f[2], f[3]);
+                        for (int c = 0; c < 4; ++c) accg[r][nt][c] = 0.f;
                     }
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt)
-                        mma_bf16_16816(acc[r][nt], a[0], a[1], a[2], a[3], xb[nt][2 * i], xb[nt][2 * i + 1]);
                 }
             }
         }
+        __syncwarp();
+        if (lane == 0 && i + D < my_steps) {
+            mbar_expect_tx(bar0 + 8 * d, STAGE_BYTES);
+            tma_load_2d(st, &wmap, bar0 + 8 * d, (s_begin + i + D) * 128, n0);
+        }
     }
-
-    reduce_and_store<NT, R, OUT_F32>(acc, red, n0, N, rows, idx, Y);
+    // (a wait that ran out has already lasted far longer than any copy takes: nothing is in flight)
+    __syncwarp();
+    // this warp's partial sums go to the start of its own (now idle) stage memory
+    float *red = reinterpret_cast<float *>(smem_raw);
+    reduce_and_store<BITS, NT, R, D * STAGE_BYTES / 4, OUT_F32>(acc, red, n0, N, rows, idx, Y);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -390,7 +433,7 @@ decode_dense_kernel(const uint16_t *__restrict__ X, int M, const int32_t *__rest
                                    cur[r][1][i].w, xv[nt][i].z, xv[nt][i].w);
                 }
     }
-    reduce_and_store<NT, R, OUT_F32>(acc, red, n0, N, rows, idx, Y);
+    reduce_and_store<0, NT, R, 16 * R * 8 * NT, OUT_F32>(acc, red, n0, N, rows, idx, Y);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -467,33 +510,51 @@ dmr_status_t set_smem(KernelT kernel, size_t bytes) {
     return DMR_OK;
 }
 
-template <int BITS, int NT, int R>
+template <int R>
+constexpr int stages_for() { return R == 1 ? 4 : (R == 2 ? 3 : 2); }
+
+template <int BITS, int NT, int R, int UNIT>
 dmr_status_t launch_lowbit_t(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
                              const uint16_t *scales, const uint8_t *zeros, int N, int K, int g, void *Y,
-                             dmr_out_t out, cudaStream_t st) {
-    const size_t smem = (size_t)kWarps * 16 * R * 8 * NT * sizeof(float);
-    const int grid = (N + 16 * R - 1) / (16 * R);
+                             dmr_out_t out, int32_t *status, cudaStream_t st) {
+    constexpr int D = stages_for<R>();
+    constexpr int ROWS = 16 * R;
+    const size_t smem = (size_t)kWarps * D * ROWS * 128 + (size_t)kWarps * D * 8;
+    const int grid = (N + ROWS - 1) / ROWS;
+    CUtensorMap wmap;
+    const uint64_t row_bytes = (uint64_t)K * BITS / 8;
+    if (!make_tensor_map_2d(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qweight, (uint64_t)N, row_bytes, row_bytes, ROWS,
+                            128, TmaSwizzle::k128B))
+        return DMR_ERR_CUDA;
     if (out == DMR_OUT_F32) {
-        auto k = decode_lowbit_kernel<BITS, NT, R, true>;
+        auto k = decode_lowbit_kernel<BITS, NT, R, UNIT, D, true>;
         if (set_smem(k, smem) != DMR_OK) return DMR_ERR_CUDA;
-        k<<<grid, kThreads, smem, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+        k<<<grid, kThreads, smem, st>>>(wmap, X, M, sel.idx, sel.count, sel.offset, scales, zeros, N, K, g, Y, status);
     } else {
-        auto k = decode_lowbit_kernel<BITS, NT, R, false>;
+        auto k = decode_lowbit_kernel<BITS, NT, R, UNIT, D, false>;
         if (set_smem(k, smem) != DMR_OK) return DMR_ERR_CUDA;
-        k<<<grid, kThreads, smem, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+        k<<<grid, kThreads, smem, st>>>(wmap, X, M, sel.idx, sel.count, sel.offset, scales, zeros, N, K, g, Y, status);
     }
     return check_launch();
 }
 
-template <int BITS, int NT>
+template <int BITS, int NT, int UNIT>
 dmr_status_t launch_lowbit_r(int R, const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
                              const uint16_t *scales, const uint8_t *zeros, int N, int K, int g, void *Y,
-                             dmr_out_t out, cudaStream_t st) {
+                             dmr_out_t out, int32_t *status, cudaStream_t st) {
     switch (R) {
-        case 4: return launch_lowbit_t<BITS, NT, 4>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
-        case 2: return launch_lowbit_t<BITS, NT, 2>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
-        default: return launch_lowbit_t<BITS, NT, 1>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+        case 4: return launch_lowbit_t<BITS, NT, 4, UNIT>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
+        case 2: return launch_lowbit_t<BITS, NT, 2, UNIT>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
+        default: return launch_lowbit_t<BITS, NT, 1, UNIT>(X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
     }
+}
+
+template <int BITS, int UNIT>
+dmr_status_t launch_lowbit_nt(int R, const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
+                              const uint16_t *scales, const uint8_t *zeros, int N, int K, int g, void *Y,
+                              dmr_out_t out, int32_t *status, cudaStream_t st) {
+    if (M <= 8) return launch_lowbit_r<BITS, 1, UNIT>(R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
+    return launch_lowbit_r<BITS, 2, UNIT>(R > 2 ? 2 : R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
 }
 
 template <int NT, int R>
@@ -515,21 +576,27 @@ dmr_status_t launch_dense_t(const uint16_t *X, int M, RowSel sel, const uint16_t
 
 }  // namespace
 
+// The unit of k a warp consumes at a time: a whole 128-wide group (or a 128-wide part of a longer
+// one), else 64.
+static int unit_for(int g) { return g % 128 == 0 ? 128 : (g % 64 == 0 ? 64 : 0); }
+
 bool decode_lowbit_supported(int M, int N, int K, int bits, int g) {
     (void)N;
-    return M >= 1 && M <= 16 && K % 128 == 0 && g % 32 == 0 && (bits == 4 || bits == 8);
+    const int unit = unit_for(g);
+    return M >= 1 && M <= 16 && unit != 0 && K % unit == 0 && (bits == 4 || bits == 8);
 }
 
 dmr_status_t launch_decode_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
                                   const uint16_t *scales, const uint8_t *zeros, int N, int K, int bits,
-                                  int g, void *Y, dmr_out_t out, cudaStream_t st) {
+                                  int g, void *Y, dmr_out_t out, int32_t *status, cudaStream_t st) {
     const int R = pick_r(N);
+    const int unit = unit_for(g);
     if (bits == 4) {
-        if (M <= 8) return launch_lowbit_r<4, 1>(R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
-        return launch_lowbit_r<4, 2>(R > 2 ? 2 : R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+        if (unit == 128) return launch_lowbit_nt<4, 128>(R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
+        return launch_lowbit_nt<4, 64>(R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
     }
-    if (M <= 8) return launch_lowbit_r<8, 1>(R > 2 ? 2 : R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
-    return launch_lowbit_r<8, 2>(R > 2 ? 2 : R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, st);
+    if (unit == 128) return launch_lowbit_nt<8, 128>(R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
+    return launch_lowbit_nt<8, 64>(R, X, M, sel, qweight, scales, zeros, N, K, g, Y, out, status, st);
 }
 
 bool decode_dense_supported(int M, int N, int K) {

@@ -137,8 +137,13 @@ def test_config1_lowbit_linear(M):
     (16, 328, 512, 8, 128),
     (1, 24, 128, 4, 128),      # smallest K the decode kernel takes
     (2, 40, 160, 4, 32),       # K not a multiple of 128: any-shape kernel
-    (40, 300, 512, 4, 128),    # M above the decode limit
+    (40, 300, 512, 4, 128),    # M above the decode limit: tensor-core GEMM, ragged N and M
     (33, 136, 384, 8, 0),
+    (64, 256, 4096, 4, 128),   # few tiles, long K: split-K with ordered reduction
+    (130, 264, 1024, 4, 64),   # two column blocks, g = 64
+    (100, 200, 2048, 8, 0),    # INT8 per-channel: one group spans all of K
+    (300, 520, 640, 4, 128),
+    (257, 128, 256, 4, 0),
 ])
 def test_lowbit_linear_shapes(M, N, K, bits, group):
     run_lowbit_case(M, N, K, bits, group, seed=3)
@@ -149,7 +154,8 @@ def test_lowbit_linear_with_outlier_channels():
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 512, 512), (4, 512, 512), (16, 1000, 1024), (11, 72, 4096),
-                                   (3, 40, 200), (40, 300, 512)])
+                                   (3, 40, 200), (40, 300, 512), (64, 256, 4096), (200, 264, 1024),
+                                   (300, 520, 640), (1000, 130, 192)])
 def test_dense_linear(M, N, K):
     W = inputs.weights(N, K, seed=6, index=N)
     X = inputs.activations(M, K, seed=6, index=M)
@@ -182,14 +188,14 @@ def test_one_hot_activations_pick_single_weights():
     N, K = 64, 512
     W = inputs.weights(N, K, seed=8)
     q, ref = quantize_both(W, 4, 128)
-    _, Wb = oracle.dequantize(*ref, K, bits=4, group=128)
+    What, _ = oracle.dequantize(*ref, K, bits=4, group=128)
     Xf = np.zeros((8, K))
     cols = [0, 1, 5, 127, 128, 300, 510, 511]
     for m, c in enumerate(cols):
         Xf[m, c] = 1.0
     Y = dmr.dmr_lowbit_linear(to_dev_bf16(inputs.f64_to_bf16_bits(Xf)), q, OUT_F32).cpu().numpy()
-    want = inputs.bf16_bits_to_f64(Wb)[:, cols].T
-    assert np.array_equal(Y.astype(np.float64), want)
+    # the kernel multiplies exact integers q - zero and scales the group sum in fp32: no rounding at all
+    assert np.array_equal(Y.astype(np.float64), What[:, cols].T)
 
 
 # ---------------- routing ----------------
