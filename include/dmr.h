@@ -69,7 +69,10 @@ size_t dmr_scales_bytes(int N, int K, dmr_qformat_t f);
 size_t dmr_zeros_bytes(int N, int K, dmr_qformat_t f);
 
 /* Scratch bytes `op` needs for these sizes (split-K partial sums, routed row lists and
- * compacted activations, a status word).  Always a multiple of 256; never 0. */
+ * compacted activations, decode counters, a status word).  Always a multiple of 256; never 0.
+ * The workspace must be zero-filled once before its first use; every call leaves the words that
+ * have to be zero (counters, status) zero again, so it can be reused without clearing.  Calls
+ * that may overlap on the GPU need separate workspaces. */
 size_t dmr_workspace_bytes(dmr_op_t op, int M, int N, int K, dmr_qformat_t f);
 
 /*

@@ -16,11 +16,13 @@ namespace {
 //   routed:    counts {n_high, n_low} (256 B), idx_high [M], idx_low [M]
 //   routed, tensor-core path: gathered activations of the low rows [M][K], then of the high rows
 //   split-K:   fp32 partial sums [splits][M][N] (shared by the two halves of a routed call)
+//   decode:    feature-group counters and per-CTA partial sums of the streaming kernel
 struct Scratch {
     int32_t *status = nullptr;
     int32_t *counts = nullptr, *idx_high = nullptr, *idx_low = nullptr;
     uint16_t *xg_low = nullptr, *xg_high = nullptr;
     float *partial = nullptr;
+    void *stream_scratch = nullptr;  // counters + partial sums of the streaming decode kernel
     size_t bytes = 0;
 };
 
@@ -60,6 +62,12 @@ Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f
         s.partial = reinterpret_cast<float *>(base + off);
         off += round_up(partial, 256);
     }
+    const bool low_stream = op != DMR_OP_DENSE_LINEAR && !low_gemm;
+    const bool dense_stream = op != DMR_OP_LOWBIT_LINEAR && !dense_gemm;
+    if (low_stream || dense_stream) {
+        s.stream_scratch = base + off;
+        off += round_up(stream_scratch_bytes(N), 256);
+    }
     s.bytes = round_up(off, 256);
     return s;
 }
@@ -89,7 +97,7 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
         }
         return launch_gemm(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.partial, ws.status, st);
     }
-    if (!decode_lowbit_supported(M < 16 ? M : 16, N, K, f.bits, g))
+    if (!stream_supported(M < 16 ? M : 16, N, K, f.bits, g))
         return launch_simple_lowbit(X, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, st);
     for (int m0 = 0; m0 < M; m0 += 16) {
         const int mc = M - m0 < 16 ? M - m0 : 16;
@@ -103,7 +111,8 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
             Xc = X + (size_t)m0 * K;
             Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
         }
-        dmr_status_t r = launch_decode_lowbit(Xc, mc, s, qweight, scales, zeros, N, K, f.bits, g, Yc, out, ws.status, st);
+        dmr_status_t r = launch_stream(Xc, mc, s, qweight, scales, zeros, N, K, f.bits, g, Yc, out, ws.stream_scratch,
+                                       ws.status, st);
         if (r != DMR_OK) return r;
     }
     return DMR_OK;
@@ -121,7 +130,7 @@ dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, 
         }
         return launch_gemm(Xin, M, sel, W, nullptr, nullptr, N, K, 0, K, Y, out, ws.partial, ws.status, st);
     }
-    if (!decode_dense_supported(M < 16 ? M : 16, N, K)) return launch_simple_dense(X, M, sel, W, N, K, Y, out, st);
+    if (!stream_supported(M < 16 ? M : 16, N, K, 16, K)) return launch_simple_dense(X, M, sel, W, N, K, Y, out, st);
     for (int m0 = 0; m0 < M; m0 += 16) {
         const int mc = M - m0 < 16 ? M - m0 : 16;
         RowSel s = sel;
@@ -134,7 +143,7 @@ dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, 
             Xc = X + (size_t)m0 * K;
             Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
         }
-        dmr_status_t r = launch_decode_dense(Xc, mc, s, W, N, K, Yc, out, st);
+        dmr_status_t r = launch_stream(Xc, mc, s, W, nullptr, nullptr, N, K, 16, K, Yc, out, ws.stream_scratch, ws.status, st);
         if (r != DMR_OK) return r;
     }
     return DMR_OK;

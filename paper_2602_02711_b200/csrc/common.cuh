@@ -60,15 +60,15 @@ dmr_status_t launch_dequantize(const uint32_t *qweight, const uint16_t *scales, 
                                int N, int K, int bits, int g, void *W_out, dmr_out_t out,
                                cudaStream_t st);
 
-// Decode family (M <= 16): tensor-core GEMV streaming the weights once.
-bool decode_lowbit_supported(int M, int N, int K, int bits, int g);
-dmr_status_t launch_decode_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,
-                                  const uint16_t *scales, const uint8_t *zeros, int N, int K,
-                                  int bits, int g, void *Y, dmr_out_t out, int32_t *status,
-                                  cudaStream_t st);
-bool decode_dense_supported(int M, int N, int K);
-dmr_status_t launch_decode_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, int N,
-                                 int K, void *Y, dmr_out_t out, cudaStream_t st);
+// Streaming decode kernel (M <= 16): persistent, one CTA per SM, weights read once.  `bits` is 4 or 8
+// for packed codes and 16 for bf16 weights.  `scratch` holds stream_scratch_bytes(N) bytes that are
+// zero before the first use (the kernel leaves its counters zeroed again).
+constexpr int kMaxStreamCtas = 256;
+size_t stream_scratch_bytes(int N);
+bool stream_supported(int M, int N, int K, int bits, int g);
+dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,
+                           const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
+                           void *scratch, int32_t *status, cudaStream_t st);
 
 // Tensor-core GEMM family (M > 16): tcgen05 MMA with TMA-staged operands.
 struct GemmPlan {

@@ -1,0 +1,686 @@
+// Decode-time linear layers (M <= 16 rows): one persistent kernel that streams the weight matrix
+// exactly once at memory speed.  Decoding re-streams the model weights for every generated token
+// and is limited by memory bandwidth, which is where weight-only quantization pays (App.
+// "Evaluation protocol", discussion of output length; App. "Latency coefficients").
+//
+// Work decomposition.  The weight matrix is cut into steps of [128 features x 128 bytes] (256
+// 4-bit codes, 128 8-bit codes or 64 bf16 weights per feature).  Steps are numbered feature-group
+// major, k minor, and CTA c of the (at most one per SM) grid takes the contiguous range
+// [c * total / ctas, (c + 1) * total / ctas): every SM streams the same number of bytes whatever
+// the shape.  A feature group whose steps are shared by several CTAs is finished by the last of
+// them to arrive, which adds the partial sums in CTA order (no floating-point atomics), so the
+// summation order of an output depends on (N, K) and the SM count only - never on M, on the
+// row's position in the batch or on the other rows.
+//
+// Inside a CTA one producer warp keeps a ring of stages full: the weight box by TMA
+// (cp.async.bulk.tensor, 128-byte swizzle) and the matching activation slice by 16-byte
+// cp.async (which also gathers the rows of a routed batch), both completing on the stage's
+// mbarrier.  Eight consumer warps each own 32 features and one half of the step's k range; the
+// product runs on the tensor cores with the weights as the 16-row operand of mma.m16n8k16 and up
+// to 8 (or 2 x 8) activation rows as the 8-column operand.  4-bit codes are unpacked with one
+// LOP3 per two codes ((w >> 4p) & 0x000F000F | 0x43004300 = {128 + q_p, 128 + q_{p+4}} as two
+// bf16) and one packed subtract of (128 + zero): the tensor-core operand is the exact integer
+// q - zero.  Products are accumulated per quantization group in fp32 and the group's scale is
+// applied to the group sum, so no weight is ever rounded: the only error against exact arithmetic
+// is fp32 summation.
+//
+// Programmatic dependent launch: the kernel lets its successor start at once and prefetches its
+// own first weight stages before waiting for its predecessor, because weights never depend on
+// the previous kernel; activations, row lists and the scratch area are touched only afterwards.
+#include <cuda_bf16.h>
+
+#include "sm100.cuh"
+
+namespace dmr {
+
+namespace {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
+constexpr int kTileRows = 128;                              // features per step
+constexpr int kStepBytes = kTileRows * 128;                 // weight bytes per step (16 KB)
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));  // (a & b) | c
+    return r;
+}
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t bf16x2_sub(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+
+// One arrival on `bar` once every cp.async issued so far by this thread has landed.
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ float ld_cg_f32(const float *p) {
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+
+// Fragment row g of a 16-row tile holds tile row tile_row_of(g) (and that + 8): rows 0,4,1,5,...
+// so that the eight lanes of one shared-memory phase (two values of g, four 16-byte chunks each)
+// land on different bank groups under the 128-byte swizzle.
+__device__ __forceinline__ int tile_row_of(int g) { return (g >> 1) | ((g & 1) << 2); }
+
+// Geometry of one step for a weight width.
+template <int BITS>
+struct StepGeom {
+    static constexpr int STEP_K = 1024 / BITS;         // weights per 128-byte row: 256, 128, 64
+    static constexpr int UNIT_K = STEP_K / 2;          // per k-half warp: 128, 64, 32
+    static constexpr int X_ROW_BYTES = STEP_K * 2;     // activation bytes per row per step
+    static constexpr int X_CHUNKS = X_ROW_BYTES / 16;  // 32, 16, 8
+};
+
+// Where 16-byte chunk c of activation row `slot` sits inside that row of a stage.  Lane (g, t) reads
+// consecutive chunks of row g starting at (its k half) * X_CHUNKS / 2 + t * (chunks per lane); the
+// permutation makes the eight lanes of a shared-memory phase (two rows, four values of t) hit
+// eight different bank groups.
+template <int BITS>
+__device__ __forceinline__ int x_chunk_pos(int c, int slot) {
+    if (BITS == 4) return c ^ (((c >> 3) & 1) << 1) ^ (slot & 1);
+    if (BITS == 8) return c ^ (slot & 1);
+    return c ^ ((slot & 1) << 2);
+}
+
+struct StreamArgs {
+    const uint16_t *X;        // [*][K] bf16
+    const int32_t *idx;       // routed: row of X / Y for batch slot s (nullptr = identity)
+    const int32_t *count;     // routed: valid slots in the list (nullptr = M)
+    const uint16_t *scales;   // low-bit only
+    const uint8_t *zeros;     // low-bit only
+    void *Y;
+    float *partial;           // [ctas][2][16 slots][128 features] fp32
+    int32_t *counters;        // [feature groups], zero on entry and on exit
+    int32_t *status;
+    int M, coff, N, K, g_size;
+    int steps_per_group;      // ceil(K / STEP_K)
+    int total_steps;          // feature groups * steps_per_group
+};
+
+__device__ __forceinline__ long long range_begin(int c, int ctas, int total) {
+    return ((long long)c * total) / ctas;
+}
+
+// Consumer-warp barrier on an mbarrier (one arrival per warp) so that the wait is bounded.
+__device__ __forceinline__ bool consumer_sync(uint32_t bar, uint32_t &phase, int32_t *status) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+    const bool ok = mbar_wait(bar, phase, status);
+    phase ^= 1u;
+    return ok;
+}
+
+template <int BITS, int NT, int GS>
+struct StreamCfg {
+    using G = StepGeom<BITS>;
+    static constexpr int SLOTS = NT * 8;
+    static constexpr int X_STAGE = SLOTS * G::X_ROW_BYTES;
+    static constexpr int STAGE = kStepBytes + X_STAGE;
+    static constexpr int D_RAW = (100 * 1024) / STAGE;
+    static constexpr int D = D_RAW > 6 ? 6 : D_RAW;
+    static constexpr int SCRATCH = SLOTS * kTileRows * 4;
+    static constexpr int BAR_OFF = D * STAGE + SCRATCH;
+    static constexpr size_t SMEM = (size_t)BAR_OFF + 256 + 1024 /*alignment slack*/;
+};
+
+// BITS: 4 / 8 = packed codes, 16 = bf16 weights.  NT: 8-row activation tiles (1 or 2).
+// GS: quantization groups per 128-code unit (2 only for 4-bit codes with 64-wide groups).
+template <int BITS, int NT, int GS, bool OUT_F32>
+__global__ void __launch_bounds__(kStreamThreads, 1)
+decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs a) {
+    using Cfg = StreamCfg<BITS, NT, GS>;
+    using Geo = StepGeom<BITS>;
+    constexpr int D = Cfg::D, SLOTS = Cfg::SLOTS, R = 2;
+    constexpr bool LOWBIT = BITS != 16;
+    constexpr int WPS = 4 / GS;  // 32-bit code words per lane, feature and group part
+    extern __shared__ uint8_t smem_dyn[];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+    auto w_stage = [&](int d) { return base + (uint32_t)d * kStepBytes; };
+    auto x_stage = [&](int d) { return base + (uint32_t)D * kStepBytes + (uint32_t)d * Cfg::X_STAGE; };
+    float *scratch = reinterpret_cast<float *>(base_ptr + D * Cfg::STAGE);
+    const uint32_t bar0 = base + Cfg::BAR_OFF;
+    auto full_bar = [&](int d) { return bar0 + 8u * d; };
+    auto empty_bar = [&](int d) { return bar0 + 64u + 8u * d; };
+    const uint32_t cons_bar = bar0 + 128u;
+    volatile int32_t *flag = reinterpret_cast<volatile int32_t *>(base_ptr + Cfg::BAR_OFF + 192);
+
+    const int ctas = gridDim.x, cta = blockIdx.x;
+    const int SPG = a.steps_per_group;
+    const int beg = (int)range_begin(cta, ctas, a.total_steps);
+    const int end = (int)range_begin(cta + 1, ctas, a.total_steps);
+    const int nsteps = end - beg;
+    const int G = LOWBIT ? a.K / a.g_size : 1;
+
+    if (threadIdx.x == 0) {
+        for (int d = 0; d < D; ++d) {
+            mbar_init(full_bar(d), 1 + 32);
+            mbar_init(empty_bar(d), kConsumerWarps);
+        }
+        mbar_init(cons_bar, kConsumerWarps);
+        fence_barrier_init();
+        prefetch_tensor_map(&wmap);
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    if (warp == kConsumerWarps) {
+        // ======================= producer warp =======================
+        // Weights never depend on the preceding kernel: start them before waiting for it
+        // (a routed call must first learn whether it has any row at all).
+        int npre = 0;
+        if (a.count == nullptr && lane == 0) {
+            for (; npre < D && npre < nsteps; ++npre) {
+                const int s = beg + npre;
+                mbar_expect_tx(full_bar(npre), kStepBytes);
+                tma_load_2d(w_stage(npre), &wmap, full_bar(npre), (s % SPG) * 128, (s / SPG) * kTileRows);
+            }
+        }
+        npre = __shfl_sync(0xFFFFFFFFu, npre, 0);
+        pdl_wait();
+        const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
+        if (rows <= 0) return;
+        // batch slot -> row of X (lane l holds slot l)
+        int my_row = -1;
+        if (lane < SLOTS && lane < rows) my_row = a.idx ? a.idx[lane] : lane;
+        int last_pf_group = -1, last_pf_rg = -1;
+        for (int i = 0; i < nsteps; ++i) {
+            const int d = i % D;
+            if (i >= D && !mbar_wait(empty_bar(d), (uint32_t)(((i / D) - 1) & 1), a.status)) break;
+            const int s = beg + i, rg = s / SPG, ks = s % SPG;
+            if (i >= npre && lane == 0) {
+                mbar_expect_tx(full_bar(d), kStepBytes);
+                tma_load_2d(w_stage(d), &wmap, full_bar(d), ks * 128, rg * kTileRows);
+            }
+            // activations of this k range, all batch slots
+            const uint32_t xs = x_stage(d);
+#pragma unroll
+            for (int it = 0; it < SLOTS * Geo::X_CHUNKS / 32; ++it) {
+                const int ch = it * 32 + lane;
+                const int slot = ch / Geo::X_CHUNKS, cc = ch % Geo::X_CHUNKS;
+                const int row = __shfl_sync(0xFFFFFFFFu, my_row, slot);
+                const int k = ks * Geo::STEP_K + cc * 8;
+                const bool valid = row >= 0 && k < a.K;
+                const uint16_t *src = valid ? a.X + (size_t)row * a.K + k : a.X;
+                cp_async16(xs + slot * Geo::X_ROW_BYTES + x_chunk_pos<BITS>(cc, slot) * 16, src, valid ? 16u : 0u);
+            }
+            cp_async_arrive(full_bar(d));
+            if (LOWBIT) {
+                // pull the scale / zero sectors of the groups ahead into L2 before the consumers ask
+                const int g0 = (ks * Geo::STEP_K) / a.g_size;
+                if (rg != last_pf_rg || g0 >= last_pf_group + 16) {
+                    last_pf_rg = rg;
+                    last_pf_group = g0;
+                    const int g1 = min(G - 1, g0 + 15);
+#pragma unroll
+                    for (int q = 0; q < kTileRows / 32; ++q) {
+                        const int n = min(rg * kTileRows + q * 32 + lane, a.N - 1);
+                        prefetch_l2(a.scales + (size_t)n * G + g0);
+                        prefetch_l2(a.scales + (size_t)n * G + g1);
+                        prefetch_l2(a.zeros + (size_t)n * G + g0);
+                        prefetch_l2(a.zeros + (size_t)n * G + g1);
+                    }
+                }
+            }
+        }
+        return;
+    }
+
+    // ======================= consumer warps =======================
+    pdl_wait();
+    const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
+    if (rows <= 0) return;
+    const int rb = warp & 3, kh = warp >> 2;     // 32-feature block, k half
+    const int g = lane >> 2, t = lane & 3;
+    const int trow = tile_row_of(g);
+    // byte offsets of this lane's code chunks inside a weight stage: features rb*32 + r*16 + trow (+8)
+    uint32_t w_off[R][2];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) w_off[r][h] = (uint32_t)((rb * 32 + r * 16 + trow + 8 * h) * 128);
+    // activation rows of this lane's fragment columns
+    uint32_t x_off[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) x_off[nt] = (uint32_t)((nt * 8 + g) * Geo::X_ROW_BYTES);
+
+    float acc[R][NT][4], accg[R][NT][4];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[r][nt][c] = accg[r][nt][c] = 0.f;
+
+    // scale / zero of (feature, group) for the current and the next step, as loaded
+    uint32_t sz_cur[R][2][GS][2], sz_nxt[R][2][GS][2];
+    auto load_sz = [&](int s, uint32_t (&dst)[R][2][GS][2]) {
+        if (!LOWBIT) return;
+        const int rg = s / SPG, ks = s % SPG;
+        const int k0 = ks * Geo::STEP_K + kh * Geo::UNIT_K;
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int n = min(rg * kTileRows + rb * 32 + r * 16 + trow + 8 * h, a.N - 1);
+#pragma unroll
+                for (int sg = 0; sg < GS; ++sg) {
+                    const int grp = min((k0 + sg * (Geo::UNIT_K / GS)) / a.g_size, G - 1);
+                    dst[r][h][sg][0] = __ldg(a.scales + (size_t)n * G + grp);
+                    dst[r][h][sg][1] = __ldg(a.zeros + (size_t)n * G + grp);
+                }
+            }
+    };
+    if (nsteps > 0) load_sz(beg, sz_nxt);
+
+    uint32_t cons_phase = 0;
+    int first_ks = -1;  // k step at which this CTA entered the current feature group
+    bool ok = true;
+    for (int i = 0; i < nsteps && ok; ++i) {
+        const int d = i % D;
+        const int s = beg + i, rg = s / SPG, ks = s % SPG;
+        if (first_ks < 0) first_ks = ks;
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int sg = 0; sg < GS; ++sg) {
+                    sz_cur[r][h][sg][0] = sz_nxt[r][h][sg][0];
+                    sz_cur[r][h][sg][1] = sz_nxt[r][h][sg][1];
+                }
+        if (i + 1 < nsteps) load_sz(s + 1, sz_nxt);
+        ok = mbar_wait(full_bar(d), (uint32_t)((i / D) & 1), a.status);
+        if (!ok) break;
+        const int k0 = ks * Geo::STEP_K + kh * Geo::UNIT_K;
+        if (k0 < a.K) {  // warp-uniform: the unit may lie past the end of a ragged row
+            const uint32_t ws = w_stage(d), xs = x_stage(d);
+#pragma unroll
+            for (int sg = 0; sg < GS; ++sg) {
+                // ---- this lane's activations, 32-bit words in k order ----
+                constexpr int XW = BITS == 4 ? 4 * WPS : (BITS == 8 ? 8 : 4);
+                uint32_t xw[NT][XW];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int i4 = 0; i4 < XW / 4; ++i4) {
+                        int c;
+                        if (BITS == 4) c = GS == 1 ? kh * 16 + t * 4 + i4 : kh * 16 + sg * 8 + t * 2 + i4;
+                        else if (BITS == 8) c = kh * 8 + t * 2 + i4;
+                        else c = kh * 4 + t;
+                        const uint4 v = lds128(xs + x_off[nt] + (uint32_t)(x_chunk_pos<BITS>(c, g) * 16));
+                        xw[nt][4 * i4 + 0] = v.x;
+                        xw[nt][4 * i4 + 1] = v.y;
+                        xw[nt][4 * i4 + 2] = v.z;
+                        xw[nt][4 * i4 + 3] = v.w;
+                    }
+                // ---- this lane's weights: WPS (4-bit) or 4 words per feature ----
+                constexpr int WW = BITS == 4 ? WPS : 4;
+                uint32_t wq[R][2][WW];
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (BITS == 4 && GS == 2) {
+                            const uint32_t chunk = (uint32_t)(kh * 4 + sg * 2 + (t >> 1)) ^ (uint32_t)trow;
+                            const uint2 v = lds64(ws + w_off[r][h] + (chunk << 4) + (uint32_t)((t & 1) * 8));
+                            wq[r][h][0] = v.x;
+                            wq[r][h][WW - 1] = v.y;
+                        } else {
+                            const uint32_t chunk = (uint32_t)(kh * 4 + t) ^ (uint32_t)trow;
+                            const uint4 v = lds128(ws + w_off[r][h] + (chunk << 4));
+                            wq[r][h][0] = v.x;
+                            wq[r][h][1 % WW] = v.y;
+                            wq[r][h][2 % WW] = v.z;
+                            wq[r][h][3 % WW] = v.w;
+                        }
+                    }
+                if (BITS == 4) {
+                    uint32_t zoff[R][2];
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t zz = 0x4300u | sz_cur[r][h][sg][1];  // bf16 of 128 + zero (exact)
+                            zoff[r][h] = zz | (zz << 16);
+                        }
+#pragma unroll
+                    for (int w = 0; w < WW; ++w)
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            // activations in unpack order: (x_p, x_{p+4}) and (x_{p+1}, x_{p+5}), p = 2 hh
+                            uint32_t b0[NT], b1[NT];
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                const uint32_t r0 = xw[nt][4 * w + hh], r2 = xw[nt][4 * w + 2 + hh];
+                                b0[nt] = prmt(r0, r2, 0x5410);
+                                b1[nt] = prmt(r0, r2, 0x7632);
+                            }
+#pragma unroll
+                            for (int r = 0; r < R; ++r) {
+                                uint32_t av[4];
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const uint32_t uu = wq[r][h][w];
+                                    const uint32_t v0 = lop3_and_or(uu >> (8 * hh), 0x000F000Fu, 0x43004300u);
+                                    const uint32_t v1 = lop3_and_or(uu >> (8 * hh + 4), 0x000F000Fu, 0x43004300u);
+                                    av[h] = bf16x2_sub(v0, zoff[r][h]);      // codes p, p+4 minus zero
+                                    av[2 + h] = bf16x2_sub(v1, zoff[r][h]);  // codes p+1, p+5
+                                }
+#pragma unroll
+                                for (int nt = 0; nt < NT; ++nt)
+                                    mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], b0[nt], b1[nt]);
+                            }
+                        }
+                } else if (BITS == 8) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        float zf[2];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) zf[h] = __uint_as_float(0x4B000000u | sz_cur[r][h][sg][1]);  // 2^23 + zero
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            uint32_t av[4];
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const uint32_t uu = wq[r][h][w];
+                                float f[4];
+#pragma unroll
+                                for (int b = 0; b < 4; ++b)  // (2^23 + byte) - (2^23 + zero) = q - zero exactly
+                                    f[b] = __fsub_rn(__uint_as_float(prmt(uu, 0x4B000000u, 0x7650u + (uint32_t)b)), zf[h]);
+                                av[h] = pack_bf16x2_rn(f[0], f[1]);  // |q - zero| <= 255: exact in bf16
+                                av[2 + h] = pack_bf16x2_rn(f[2], f[3]);
+                            }
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt)
+                                mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], xw[nt][2 * w], xw[nt][2 * w + 1]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int p = 0; p < 2; ++p)
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt)
+                                mma_bf16_16816(acc[r][nt], wq[r][0][2 * p], wq[r][1][2 * p], wq[r][0][2 * p + 1],
+                                               wq[r][1][2 * p + 1], xw[nt][2 * p], xw[nt][2 * p + 1]);
+                }
+                if (LOWBIT) {
+                    // the group sum is complete for this warp when its next unit (one step further)
+                    // lies in another group, in another feature group or outside this CTA's range
+                    const int kpart = k0 + sg * (Geo::UNIT_K / GS);
+                    const int grp = kpart / a.g_size;
+                    const bool closes = GS == 2 || (kpart + Geo::STEP_K) / a.g_size != grp || ks == SPG - 1 ||
+                                        i == nsteps - 1 || kpart + Geo::STEP_K >= a.K;
+                    if (closes) {
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            const float s0 = __uint_as_float(sz_cur[r][0][sg][0] << 16);
+                            const float s1 = __uint_as_float(sz_cur[r][1][sg][0] << 16);
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                acc[r][nt][0] = fmaf(s0, accg[r][nt][0], acc[r][nt][0]);
+                                acc[r][nt][1] = fmaf(s0, accg[r][nt][1], acc[r][nt][1]);
+                                acc[r][nt][2] = fmaf(s1, accg[r][nt][2], acc[r][nt][2]);
+                                acc[r][nt][3] = fmaf(s1, accg[r][nt][3], acc[r][nt][3]);
+#pragma unroll
+                                for (int c = 0; c < 4; ++c) accg[r][nt][c] = 0.f;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar(d));
+
+        // ---- end of this CTA's part of the feature group: combine and write ----
+        if (ks == SPG - 1 || i == nsteps - 1) {
+            const bool complete = first_ks == 0 && ks == SPG - 1;
+            // k half 1 parks its sums, k half 0 adds them (fixed order) and parks the total
+            if (kh == 1) {
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            scratch[(nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 32 + r * 16 + trow + 8 * (c >> 1)] = acc[r][nt][c];
+            }
+            ok = consumer_sync(cons_bar, cons_phase, a.status);
+            if (!ok) break;
+            if (kh == 0) {
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            float *p = scratch + (nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 32 + r * 16 + trow + 8 * (c >> 1);
+                            *p = acc[r][nt][c] + *p;
+                        }
+            }
+            ok = consumer_sync(cons_bar, cons_phase, a.status);
+            if (!ok) break;
+            const int n_base = rg * kTileRows;
+            auto store_y = [&](int o, float v) {
+                const int slot = o / kTileRows, n = n_base + o % kTileRows;
+                if (slot >= rows || n >= a.N) return;
+                const int row = a.idx ? a.idx[slot] : slot;
+                if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
+                else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
+            };
+            if (complete) {
+                for (int o = threadIdx.x; o < SLOTS * kTileRows; o += kConsumerWarps * 32) store_y(o, scratch[o]);
+            } else {
+                // shared feature group: leave the partial sums in the scratch area; the CTA that
+                // arrives last adds all parts in CTA order and writes the result
+                const int which = beg > rg * SPG ? 0 : 1;
+                float *mine = a.partial + ((size_t)cta * 2 + which) * (16 * kTileRows);
+                for (int o = threadIdx.x; o < SLOTS * kTileRows; o += kConsumerWarps * 32) mine[o] = scratch[o];
+                __threadfence();
+                ok = consumer_sync(cons_bar, cons_phase, a.status);
+                if (!ok) break;
+                const long long s_first = (long long)rg * SPG, s_last = s_first + SPG - 1;
+                const int c_first = (int)(((s_first + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
+                const int c_last = (int)(((s_last + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
+                if (threadIdx.x == 0) {
+                    const int old = atomicAdd(a.counters + rg, 1);
+                    const int last = old == c_last - c_first;
+                    if (last) a.counters[rg] = 0;  // leave the counter ready for the next call
+                    __threadfence();
+                    *flag = last;
+                }
+                ok = consumer_sync(cons_bar, cons_phase, a.status);
+                if (!ok) break;
+                if (*flag) {
+                    for (int o = threadIdx.x; o < SLOTS * kTileRows; o += kConsumerWarps * 32) {
+                        float v = 0.f;
+                        for (int cj = c_first; cj <= c_last; ++cj) {
+                            const int wj = range_begin(cj, ctas, a.total_steps) > s_first ? 0 : 1;
+                            v += ld_cg_f32(a.partial + ((size_t)cj * 2 + wj) * (16 * kTileRows) + o);
+                        }
+                        store_y(o, v);
+                    }
+                }
+            }
+            ok = consumer_sync(cons_bar, cons_phase, a.status);  // scratch and flag are free again
+            if (!ok) break;
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) acc[r][nt][c] = 0.f;
+            first_ks = -1;
+        }
+    }
+}
+
+int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    return dev;
+}
+
+int sm_count() {
+    static int cached[64] = {};
+    const int dev = current_device();
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) cached[dev] = n;
+        else cached[dev] = 148;
+    }
+    return cached[dev];
+}
+
+template <int BITS, int NT, int GS, bool OUT_F32>
+dmr_status_t launch_stream_t(const CUtensorMap &wmap, const StreamArgs &a, int ctas, cudaStream_t st) {
+    using Cfg = StreamCfg<BITS, NT, GS>;
+    auto kernel = decode_stream_kernel<BITS, NT, GS, OUT_F32>;
+    static bool configured_on[64] = {};
+    bool &configured = configured_on[current_device()];
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            return DMR_ERR_CUDA;
+        }
+        configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas, 1, 1);
+    cfg.blockDim = dim3(kStreamThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, wmap, a);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        (void)cudaGetLastError();
+        return DMR_ERR_CUDA;
+    }
+    return check_launch();
+}
+
+template <int BITS, int GS>
+dmr_status_t launch_stream_nt(const CUtensorMap &wmap, const StreamArgs &a, int ctas, dmr_out_t out, cudaStream_t st) {
+    if (a.M <= 8) {
+        if (out == DMR_OUT_F32) return launch_stream_t<BITS, 1, GS, true>(wmap, a, ctas, st);
+        return launch_stream_t<BITS, 1, GS, false>(wmap, a, ctas, st);
+    }
+    if (out == DMR_OUT_F32) return launch_stream_t<BITS, 2, GS, true>(wmap, a, ctas, st);
+    return launch_stream_t<BITS, 2, GS, false>(wmap, a, ctas, st);
+}
+
+}  // namespace
+
+size_t stream_scratch_bytes(int N) {
+    const size_t groups = (size_t)(N + kTileRows - 1) / kTileRows;
+    return round_up(groups * sizeof(int32_t), 256) + (size_t)kMaxStreamCtas * 2 * 16 * kTileRows * sizeof(float);
+}
+
+bool stream_supported(int M, int N, int K, int bits /*16 = bf16 weights*/, int g) {
+    (void)N;
+    if (M < 1 || M > 16) return false;
+    if (bits == 16) return K % 8 == 0;
+    if (bits == 4) return g % 128 == 0 || g == 64;
+    if (bits == 8) return g % 64 == 0;
+    return false;
+}
+
+dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,
+                           const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
+                           void *scratch, int32_t *status, cudaStream_t st) {
+    const int step_k = 1024 / bits;
+    StreamArgs a;
+    a.X = X;
+    a.idx = sel.idx;
+    a.count = sel.count;
+    a.scales = scales;
+    a.zeros = zeros;
+    a.Y = Y;
+    const size_t groups = (size_t)(N + kTileRows - 1) / kTileRows;
+    a.counters = reinterpret_cast<int32_t *>(scratch);
+    a.partial = reinterpret_cast<float *>(reinterpret_cast<char *>(scratch) + round_up(groups * sizeof(int32_t), 256));
+    a.status = status;
+    a.M = M;
+    a.coff = sel.offset;
+    a.N = N;
+    a.K = K;
+    a.g_size = bits == 16 ? K : g;
+    a.steps_per_group = (K + step_k - 1) / step_k;
+    const long long total = (long long)groups * a.steps_per_group;
+    if (total > 0x7FFFFFFF) return DMR_ERR_UNSUPPORTED;
+    a.total_steps = (int)total;
+    int ctas = sm_count();
+    if (ctas > kMaxStreamCtas) ctas = kMaxStreamCtas;
+    if (ctas > a.total_steps) ctas = a.total_steps;
+    CUtensorMap wmap;
+    const uint64_t row_bytes = (uint64_t)K * bits / 8;
+    if (!make_tensor_map_2d(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, weights, (uint64_t)N, row_bytes, row_bytes, kTileRows,
+                            128, TmaSwizzle::k128B))
+        return DMR_ERR_CUDA;
+    if (bits == 16) return launch_stream_nt<16, 1>(wmap, a, ctas, out, st);
+    if (bits == 8) return launch_stream_nt<8, 1>(wmap, a, ctas, out, st);
+    if (g == 64) return launch_stream_nt<4, 2>(wmap, a, ctas, out, st);
+    return launch_stream_nt<4, 1>(wmap, a, ctas, out, st);
+}
+
+}  // namespace dmr
