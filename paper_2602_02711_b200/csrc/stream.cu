@@ -29,16 +29,25 @@
 // the previous kernel; activations, row lists and the scratch area are touched only afterwards.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "sm100.cuh"
 
 namespace dmr {
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
+constexpr int kR = 1;                                        // 16-feature tiles per consumer warp
+constexpr int kRowBlocks = 128 / (16 * kR);                  // consumer warps side by side over the features
+constexpr int kConsumerWarps = 2 * kRowBlocks;               // two k halves
 constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
 constexpr int kTileRows = 128;                              // features per step
 constexpr int kStepBytes = kTileRows * 128;                 // weight bytes per step (16 KB)
+constexpr int kMaxStages = 12;
+#ifndef DMR_STAGE_BUDGET_KB
+#define DMR_STAGE_BUDGET_KB 100
+#endif
+constexpr int kStageBudget = DMR_STAGE_BUDGET_KB;          // shared memory for the stage ring, KB
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                                uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -47,6 +56,16 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         "{%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Same product with a zero accumulator operand: c = a * b.
+__device__ __forceinline__ void mma_bf16_16816_zero(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                    uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%10,%10,%10,%10};"
+        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 
 __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
@@ -100,12 +119,6 @@ __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefe
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-__device__ __forceinline__ float ld_cg_f32(const float *p) {
-    float v;
-    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
-    return v;
-}
-
 // Fragment row g of a 16-row tile holds tile row tile_row_of(g) (and that + 8): rows 0,4,1,5,...
 // so that the eight lanes of one shared-memory phase (two values of g, four 16-byte chunks each)
 // land on different bank groups under the 128-byte swizzle.
@@ -142,6 +155,7 @@ struct StreamArgs {
     int32_t *counters;        // [feature groups], zero on entry and on exit
     int32_t *status;
     int M, coff, N, K, g_size;
+    int g_shift;              // log2(g_size) when it is a power of two, else -1
     int steps_per_group;      // ceil(K / STEP_K)
     int total_steps;          // feature groups * steps_per_group
 };
@@ -165,21 +179,22 @@ struct StreamCfg {
     static constexpr int SLOTS = NT * 8;
     static constexpr int X_STAGE = SLOTS * G::X_ROW_BYTES;
     static constexpr int STAGE = kStepBytes + X_STAGE;
-    static constexpr int D_RAW = (100 * 1024) / STAGE;
-    static constexpr int D = D_RAW > 6 ? 6 : D_RAW;
+    static constexpr int D_RAW = (kStageBudget * 1024) / STAGE;
+    static constexpr int D = D_RAW > kMaxStages ? kMaxStages : D_RAW;
     static constexpr int SCRATCH = SLOTS * kTileRows * 4;
     static constexpr int BAR_OFF = D * STAGE + SCRATCH;
-    static constexpr size_t SMEM = (size_t)BAR_OFF + 256 + 1024 /*alignment slack*/;
+    static constexpr size_t SMEM = (size_t)BAR_OFF + 512 + 1024 /*alignment slack*/;
 };
 
 // BITS: 4 / 8 = packed codes, 16 = bf16 weights.  NT: 8-row activation tiles (1 or 2).
 // GS: quantization groups per 128-code unit (2 only for 4-bit codes with 64-wide groups).
-template <int BITS, int NT, int GS, bool OUT_F32>
+// CE: every unit a warp consumes ends its quantization group (group size == unit size).
+template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
 __global__ void __launch_bounds__(kStreamThreads, 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs a) {
     using Cfg = StreamCfg<BITS, NT, GS>;
     using Geo = StepGeom<BITS>;
-    constexpr int D = Cfg::D, SLOTS = Cfg::SLOTS, R = 2;
+    constexpr int D = Cfg::D, SLOTS = Cfg::SLOTS, R = kR;
     constexpr bool LOWBIT = BITS != 16;
     constexpr int WPS = 4 / GS;  // 32-bit code words per lane, feature and group part
     extern __shared__ uint8_t smem_dyn[];
@@ -192,9 +207,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
     float *scratch = reinterpret_cast<float *>(base_ptr + D * Cfg::STAGE);
     const uint32_t bar0 = base + Cfg::BAR_OFF;
     auto full_bar = [&](int d) { return bar0 + 8u * d; };
-    auto empty_bar = [&](int d) { return bar0 + 64u + 8u * d; };
-    const uint32_t cons_bar = bar0 + 128u;
-    volatile int32_t *flag = reinterpret_cast<volatile int32_t *>(base_ptr + Cfg::BAR_OFF + 192);
+    auto empty_bar = [&](int d) { return bar0 + 128u + 8u * d; };
+    const uint32_t cons_bar = bar0 + 256u;
+    volatile int32_t *flag = reinterpret_cast<volatile int32_t *>(base_ptr + Cfg::BAR_OFF + 320);
 
     const int ctas = gridDim.x, cta = blockIdx.x;
     const int SPG = a.steps_per_group;
@@ -202,6 +217,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
     const int end = (int)range_begin(cta + 1, ctas, a.total_steps);
     const int nsteps = end - beg;
     const int G = LOWBIT ? a.K / a.g_size : 1;
+    // quantization group of input feature k without a division in the common cases
+    auto group_of_k = [&](int k) { return a.g_shift >= 0 ? (k >> a.g_shift) : (G == 1 ? 0 : k / a.g_size); };
+    const int rg_first = beg / SPG, ks_first = beg - rg_first * SPG;
 
     if (threadIdx.x == 0) {
         for (int d = 0; d < D; ++d) {
@@ -221,10 +239,14 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
         // (a routed call must first learn whether it has any row at all).
         int npre = 0;
         if (a.count == nullptr && lane == 0) {
+            int rg = rg_first, ks = ks_first;
             for (; npre < D && npre < nsteps; ++npre) {
-                const int s = beg + npre;
                 mbar_expect_tx(full_bar(npre), kStepBytes);
-                tma_load_2d(w_stage(npre), &wmap, full_bar(npre), (s % SPG) * 128, (s / SPG) * kTileRows);
+                tma_load_2d(w_stage(npre), &wmap, full_bar(npre), ks * 128, rg * kTileRows);
+                if (++ks == SPG) {
+                    ks = 0;
+                    ++rg;
+                }
             }
         }
         npre = __shfl_sync(0xFFFFFFFFu, npre, 0);
@@ -235,30 +257,36 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
         int my_row = -1;
         if (lane < SLOTS && lane < rows) my_row = a.idx ? a.idx[lane] : lane;
         int last_pf_group = -1, last_pf_rg = -1;
+        const int xchunks = rows * Geo::X_CHUNKS;  // slots past `rows` feed output columns nobody reads
+        int rg = rg_first, ks = ks_first - 1;
         for (int i = 0; i < nsteps; ++i) {
             const int d = i % D;
+            if (++ks == SPG) {
+                ks = 0;
+                ++rg;
+            }
             if (i >= D && !mbar_wait(empty_bar(d), (uint32_t)(((i / D) - 1) & 1), a.status)) break;
-            const int s = beg + i, rg = s / SPG, ks = s % SPG;
             if (i >= npre && lane == 0) {
                 mbar_expect_tx(full_bar(d), kStepBytes);
                 tma_load_2d(w_stage(d), &wmap, full_bar(d), ks * 128, rg * kTileRows);
             }
             // activations of this k range, all batch slots
             const uint32_t xs = x_stage(d);
-#pragma unroll
-            for (int it = 0; it < SLOTS * Geo::X_CHUNKS / 32; ++it) {
-                const int ch = it * 32 + lane;
+            for (int c0 = 0; c0 < xchunks; c0 += 32) {
+                const int ch = c0 + lane;
                 const int slot = ch / Geo::X_CHUNKS, cc = ch % Geo::X_CHUNKS;
-                const int row = __shfl_sync(0xFFFFFFFFu, my_row, slot);
+                const int row = __shfl_sync(0xFFFFFFFFu, my_row, slot & 31);
                 const int k = ks * Geo::STEP_K + cc * 8;
-                const bool valid = row >= 0 && k < a.K;
-                const uint16_t *src = valid ? a.X + (size_t)row * a.K + k : a.X;
-                cp_async16(xs + slot * Geo::X_ROW_BYTES + x_chunk_pos<BITS>(cc, slot) * 16, src, valid ? 16u : 0u);
+                if (ch < xchunks) {
+                    const bool valid = k < a.K;  // past the end of a ragged row: zeros
+                    const uint16_t *src = valid ? a.X + (size_t)row * a.K + k : a.X;
+                    cp_async16(xs + slot * Geo::X_ROW_BYTES + x_chunk_pos<BITS>(cc, slot) * 16, src, valid ? 16u : 0u);
+                }
             }
             cp_async_arrive(full_bar(d));
             if (LOWBIT) {
                 // pull the scale / zero sectors of the groups ahead into L2 before the consumers ask
-                const int g0 = (ks * Geo::STEP_K) / a.g_size;
+                const int g0 = group_of_k(ks * Geo::STEP_K);
                 if (rg != last_pf_rg || g0 >= last_pf_group + 16) {
                     last_pf_rg = rg;
                     last_pf_group = g0;
@@ -281,19 +309,40 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
     pdl_wait();
     const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
     if (rows <= 0) return;
-    const int rb = warp & 3, kh = warp >> 2;     // 32-feature block, k half
+    const int rb = warp % kRowBlocks, kh = warp / kRowBlocks;  // feature block, k half
     const int g = lane >> 2, t = lane & 3;
     const int trow = tile_row_of(g);
-    // byte offsets of this lane's code chunks inside a weight stage: features rb*32 + r*16 + trow (+8)
-    uint32_t w_off[R][2];
+    const int K = a.K, N = a.N;
+    // Byte offsets of this lane's code chunks inside a weight stage (features rb*16R + r*16 + trow
+    // (+8), 128-byte rows, chunk index XOR row % 8) and of its activation chunks inside an
+    // activation stage; all fixed for the lifetime of the kernel.
+    uint32_t w_off[R][2][GS];
 #pragma unroll
     for (int r = 0; r < R; ++r)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) w_off[r][h] = (uint32_t)((rb * 32 + r * 16 + trow + 8 * h) * 128);
-    // activation rows of this lane's fragment columns
-    uint32_t x_off[NT];
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) x_off[nt] = (uint32_t)((nt * 8 + g) * Geo::X_ROW_BYTES);
+            for (int sg = 0; sg < GS; ++sg) {
+                const uint32_t rowb = (uint32_t)((rb * 16 * R + r * 16 + trow + 8 * h) * 128);
+                if (BITS == 4 && GS == 2)
+                    w_off[r][h][sg] = rowb + ((((uint32_t)(kh * 4 + sg * 2 + (t >> 1))) ^ (uint32_t)trow) << 4) + (uint32_t)((t & 1) * 8);
+                else
+                    w_off[r][h][sg] = rowb + ((((uint32_t)(kh * 4 + t)) ^ (uint32_t)trow) << 4);
+            }
+    constexpr int XW = BITS == 4 ? 4 * WPS : (BITS == 8 ? 8 : 4);  // activation words per lane, token and group part
+    uint32_t x_off[NT][GS][XW / 4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int sg = 0; sg < GS; ++sg)
+#pragma unroll
+            for (int i4 = 0; i4 < XW / 4; ++i4) {
+                int c;
+                if (BITS == 4) c = GS == 1 ? kh * 16 + t * 4 + i4 : kh * 16 + sg * 8 + t * 2 + i4;
+                else if (BITS == 8) c = kh * 8 + t * 2 + i4;
+                else c = kh * 4 + t;
+                x_off[nt][sg][i4] = (uint32_t)((nt * 8 + g) * Geo::X_ROW_BYTES + x_chunk_pos<BITS>(c, g) * 16);
+            }
 
     float acc[R][NT][4], accg[R][NT][4];
 #pragma unroll
@@ -303,63 +352,53 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[r][nt][c] = accg[r][nt][c] = 0.f;
 
-    // scale / zero of (feature, group) for the current and the next step, as loaded
-    uint32_t sz_cur[R][2][GS][2], sz_nxt[R][2][GS][2];
-    auto load_sz = [&](int s, uint32_t (&dst)[R][2][GS][2]) {
+    // scale / zero of (feature, group), loaded one step ahead into one of two register sets
+    typedef uint32_t SzRegs[R][2][GS][2];
+    SzRegs sz_a, sz_b;
+    auto load_sz = [&](int rg, int ks, SzRegs &dst) {
         if (!LOWBIT) return;
-        const int rg = s / SPG, ks = s % SPG;
         const int k0 = ks * Geo::STEP_K + kh * Geo::UNIT_K;
 #pragma unroll
         for (int r = 0; r < R; ++r)
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const int n = min(rg * kTileRows + rb * 32 + r * 16 + trow + 8 * h, a.N - 1);
+                const int n = min(rg * kTileRows + rb * 16 * R + r * 16 + trow + 8 * h, N - 1);
 #pragma unroll
                 for (int sg = 0; sg < GS; ++sg) {
-                    const int grp = min((k0 + sg * (Geo::UNIT_K / GS)) / a.g_size, G - 1);
+                    const int grp = min(group_of_k(k0 + sg * (Geo::UNIT_K / GS)), G - 1);
                     dst[r][h][sg][0] = __ldg(a.scales + (size_t)n * G + grp);
                     dst[r][h][sg][1] = __ldg(a.zeros + (size_t)n * G + grp);
                 }
             }
     };
-    if (nsteps > 0) load_sz(beg, sz_nxt);
+    if (nsteps > 0) load_sz(rg_first, ks_first, sz_a);
 
     uint32_t cons_phase = 0;
     int first_ks = -1;  // k step at which this CTA entered the current feature group
-    bool ok = true;
-    for (int i = 0; i < nsteps && ok; ++i) {
+    int rg = rg_first, ks = ks_first - 1;
+
+    // One step of the ring: `cur` holds this step's scales / zeros, `nxt` receives the next step's.
+    auto do_step = [&](int i, SzRegs &cur, SzRegs &nxt) -> bool {
         const int d = i % D;
-        const int s = beg + i, rg = s / SPG, ks = s % SPG;
+        if (++ks == SPG) {
+            ks = 0;
+            ++rg;
+        }
         if (first_ks < 0) first_ks = ks;
-#pragma unroll
-        for (int r = 0; r < R; ++r)
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int sg = 0; sg < GS; ++sg) {
-                    sz_cur[r][h][sg][0] = sz_nxt[r][h][sg][0];
-                    sz_cur[r][h][sg][1] = sz_nxt[r][h][sg][1];
-                }
-        if (i + 1 < nsteps) load_sz(s + 1, sz_nxt);
-        ok = mbar_wait(full_bar(d), (uint32_t)((i / D) & 1), a.status);
-        if (!ok) break;
+        if (i + 1 < nsteps) load_sz(ks + 1 == SPG ? rg + 1 : rg, ks + 1 == SPG ? 0 : ks + 1, nxt);
+        if (!mbar_wait(full_bar(d), (uint32_t)((i / D) & 1), a.status)) return false;
         const int k0 = ks * Geo::STEP_K + kh * Geo::UNIT_K;
-        if (k0 < a.K) {  // warp-uniform: the unit may lie past the end of a ragged row
+        if (k0 < K) {  // warp-uniform: the unit may lie past the end of a ragged row
             const uint32_t ws = w_stage(d), xs = x_stage(d);
 #pragma unroll
             for (int sg = 0; sg < GS; ++sg) {
                 // ---- this lane's activations, 32-bit words in k order ----
-                constexpr int XW = BITS == 4 ? 4 * WPS : (BITS == 8 ? 8 : 4);
                 uint32_t xw[NT][XW];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                     for (int i4 = 0; i4 < XW / 4; ++i4) {
-                        int c;
-                        if (BITS == 4) c = GS == 1 ? kh * 16 + t * 4 + i4 : kh * 16 + sg * 8 + t * 2 + i4;
-                        else if (BITS == 8) c = kh * 8 + t * 2 + i4;
-                        else c = kh * 4 + t;
-                        const uint4 v = lds128(xs + x_off[nt] + (uint32_t)(x_chunk_pos<BITS>(c, g) * 16));
+                        const uint4 v = lds128(xs + x_off[nt][sg][i4]);
                         xw[nt][4 * i4 + 0] = v.x;
                         xw[nt][4 * i4 + 1] = v.y;
                         xw[nt][4 * i4 + 2] = v.z;
@@ -373,27 +412,28 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         if (BITS == 4 && GS == 2) {
-                            const uint32_t chunk = (uint32_t)(kh * 4 + sg * 2 + (t >> 1)) ^ (uint32_t)trow;
-                            const uint2 v = lds64(ws + w_off[r][h] + (chunk << 4) + (uint32_t)((t & 1) * 8));
+                            const uint2 v = lds64(ws + w_off[r][h][sg]);
                             wq[r][h][0] = v.x;
                             wq[r][h][WW - 1] = v.y;
                         } else {
-                            const uint32_t chunk = (uint32_t)(kh * 4 + t) ^ (uint32_t)trow;
-                            const uint4 v = lds128(ws + w_off[r][h] + (chunk << 4));
+                            const uint4 v = lds128(ws + w_off[r][h][sg]);
                             wq[r][h][0] = v.x;
                             wq[r][h][1 % WW] = v.y;
                             wq[r][h][2 % WW] = v.z;
                             wq[r][h][3 % WW] = v.w;
                         }
                     }
+                // When every unit ends its quantization group the group sum starts from a zero
+                // accumulator operand instead of cleared registers.
+                bool fresh = CE;
                 if (BITS == 4) {
                     uint32_t zoff[R][2];
 #pragma unroll
                     for (int r = 0; r < R; ++r)
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const uint32_t zz = 0x4300u | sz_cur[r][h][sg][1];  // bf16 of 128 + zero (exact)
-                            zoff[r][h] = zz | (zz << 16);
+                            const uint32_t zz = 0x4300u | cur[r][h][sg][1];  // bf16 of 128 + zero (exact)
+                            zoff[r][h] = prmt(zz, zz, 0x1010);
                         }
 #pragma unroll
                     for (int w = 0; w < WW; ++w)
@@ -419,33 +459,37 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
                                     av[2 + h] = bf16x2_sub(v1, zoff[r][h]);  // codes p+1, p+5
                                 }
 #pragma unroll
-                                for (int nt = 0; nt < NT; ++nt)
-                                    mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], b0[nt], b1[nt]);
+                                for (int nt = 0; nt < NT; ++nt) {
+                                    if (fresh) mma_bf16_16816_zero(accg[r][nt], av[0], av[1], av[2], av[3], b0[nt], b1[nt]);
+                                    else mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], b0[nt], b1[nt]);
+                                }
                             }
+                            fresh = false;
                         }
                 } else if (BITS == 8) {
 #pragma unroll
-                    for (int r = 0; r < R; ++r) {
-                        float zf[2];
+                    for (int w = 0; w < 4; ++w) {
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) zf[h] = __uint_as_float(0x4B000000u | sz_cur[r][h][sg][1]);  // 2^23 + zero
-#pragma unroll
-                        for (int w = 0; w < 4; ++w) {
+                        for (int r = 0; r < R; ++r) {
                             uint32_t av[4];
 #pragma unroll
                             for (int h = 0; h < 2; ++h) {
+                                const float zf = __uint_as_float(0x4B000000u | cur[r][h][sg][1]);  // 2^23 + zero
                                 const uint32_t uu = wq[r][h][w];
                                 float f[4];
 #pragma unroll
                                 for (int b = 0; b < 4; ++b)  // (2^23 + byte) - (2^23 + zero) = q - zero exactly
-                                    f[b] = __fsub_rn(__uint_as_float(prmt(uu, 0x4B000000u, 0x7650u + (uint32_t)b)), zf[h]);
+                                    f[b] = __fsub_rn(__uint_as_float(prmt(uu, 0x4B000000u, 0x7650u + (uint32_t)b)), zf);
                                 av[h] = pack_bf16x2_rn(f[0], f[1]);  // |q - zero| <= 255: exact in bf16
                                 av[2 + h] = pack_bf16x2_rn(f[2], f[3]);
                             }
 #pragma unroll
-                            for (int nt = 0; nt < NT; ++nt)
-                                mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], xw[nt][2 * w], xw[nt][2 * w + 1]);
+                            for (int nt = 0; nt < NT; ++nt) {
+                                if (fresh) mma_bf16_16816_zero(accg[r][nt], av[0], av[1], av[2], av[3], xw[nt][2 * w], xw[nt][2 * w + 1]);
+                                else mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], xw[nt][2 * w], xw[nt][2 * w + 1]);
+                            }
                         }
+                        fresh = false;
                     }
                 } else {
 #pragma unroll
@@ -461,22 +505,23 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
                     // the group sum is complete for this warp when its next unit (one step further)
                     // lies in another group, in another feature group or outside this CTA's range
                     const int kpart = k0 + sg * (Geo::UNIT_K / GS);
-                    const int grp = kpart / a.g_size;
-                    const bool closes = GS == 2 || (kpart + Geo::STEP_K) / a.g_size != grp || ks == SPG - 1 ||
-                                        i == nsteps - 1 || kpart + Geo::STEP_K >= a.K;
+                    const bool closes = CE || group_of_k(kpart + Geo::STEP_K) != group_of_k(kpart) || ks == SPG - 1 ||
+                                        i == nsteps - 1 || kpart + Geo::STEP_K >= K;
                     if (closes) {
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
-                            const float s0 = __uint_as_float(sz_cur[r][0][sg][0] << 16);
-                            const float s1 = __uint_as_float(sz_cur[r][1][sg][0] << 16);
+                            const float s0 = __uint_as_float(cur[r][0][sg][0] << 16);
+                            const float s1 = __uint_as_float(cur[r][1][sg][0] << 16);
 #pragma unroll
                             for (int nt = 0; nt < NT; ++nt) {
                                 acc[r][nt][0] = fmaf(s0, accg[r][nt][0], acc[r][nt][0]);
                                 acc[r][nt][1] = fmaf(s0, accg[r][nt][1], acc[r][nt][1]);
                                 acc[r][nt][2] = fmaf(s1, accg[r][nt][2], acc[r][nt][2]);
                                 acc[r][nt][3] = fmaf(s1, accg[r][nt][3], acc[r][nt][3]);
+                                if (!CE) {
 #pragma unroll
-                                for (int c = 0; c < 4; ++c) accg[r][nt][c] = 0.f;
+                                    for (int c = 0; c < 4; ++c) accg[r][nt][c] = 0.f;
+                                }
                             }
                         }
                     }
@@ -497,10 +542,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
                     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
-                            scratch[(nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 32 + r * 16 + trow + 8 * (c >> 1)] = acc[r][nt][c];
+                            scratch[(nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 16 * R + r * 16 + trow + 8 * (c >> 1)] = acc[r][nt][c];
             }
-            ok = consumer_sync(cons_bar, cons_phase, a.status);
-            if (!ok) break;
+            if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
             if (kh == 0) {
 #pragma unroll
                 for (int r = 0; r < R; ++r)
@@ -508,12 +552,11 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
                     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
-                            float *p = scratch + (nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 32 + r * 16 + trow + 8 * (c >> 1);
+                            float *p = scratch + (nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 16 * R + r * 16 + trow + 8 * (c >> 1);
                             *p = acc[r][nt][c] + *p;
                         }
             }
-            ok = consumer_sync(cons_bar, cons_phase, a.status);
-            if (!ok) break;
+            if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
             const int n_base = rg * kTileRows;
             auto store_y = [&](int o, float v) {
                 const int slot = o / kTileRows, n = n_base + o % kTileRows;
@@ -528,11 +571,11 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
                 // shared feature group: leave the partial sums in the scratch area; the CTA that
                 // arrives last adds all parts in CTA order and writes the result
                 const int which = beg > rg * SPG ? 0 : 1;
-                float *mine = a.partial + ((size_t)cta * 2 + which) * (16 * kTileRows);
-                for (int o = threadIdx.x; o < SLOTS * kTileRows; o += kConsumerWarps * 32) mine[o] = scratch[o];
+                float4 *mine = reinterpret_cast<float4 *>(a.partial + ((size_t)cta * 2 + which) * (16 * kTileRows));
+                for (int o4 = threadIdx.x; o4 < SLOTS * kTileRows / 4; o4 += kConsumerWarps * 32)
+                    mine[o4] = reinterpret_cast<const float4 *>(scratch)[o4];
                 __threadfence();
-                ok = consumer_sync(cons_bar, cons_phase, a.status);
-                if (!ok) break;
+                if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
                 const long long s_first = (long long)rg * SPG, s_last = s_first + SPG - 1;
                 const int c_first = (int)(((s_first + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
                 const int c_last = (int)(((s_last + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
@@ -543,21 +586,36 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
                     __threadfence();
                     *flag = last;
                 }
-                ok = consumer_sync(cons_bar, cons_phase, a.status);
-                if (!ok) break;
+                if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
                 if (*flag) {
-                    for (int o = threadIdx.x; o < SLOTS * kTileRows; o += kConsumerWarps * 32) {
-                        float v = 0.f;
-                        for (int cj = c_first; cj <= c_last; ++cj) {
-                            const int wj = range_begin(cj, ctas, a.total_steps) > s_first ? 0 : 1;
-                            v += ld_cg_f32(a.partial + ((size_t)cj * 2 + wj) * (16 * kTileRows) + o);
+                    // loads of up to eight parts are in flight together; the additions keep CTA order
+                    for (int o4 = threadIdx.x; o4 < SLOTS * kTileRows / 4; o4 += kConsumerWarps * 32) {
+                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int cj0 = c_first; cj0 <= c_last; cj0 += 8) {
+                            float4 p[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const int cj = min(cj0 + u, c_last);
+                                const int wj = range_begin(cj, ctas, a.total_steps) > s_first ? 0 : 1;
+                                p[u] = __ldcg(reinterpret_cast<const float4 *>(a.partial + ((size_t)cj * 2 + wj) * (16 * kTileRows)) + o4);
+                            }
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                if (cj0 + u <= c_last) {
+                                    v.x += p[u].x;
+                                    v.y += p[u].y;
+                                    v.z += p[u].z;
+                                    v.w += p[u].w;
+                                }
                         }
-                        store_y(o, v);
+                        store_y(4 * o4 + 0, v.x);
+                        store_y(4 * o4 + 1, v.y);
+                        store_y(4 * o4 + 2, v.z);
+                        store_y(4 * o4 + 3, v.w);
                     }
                 }
             }
-            ok = consumer_sync(cons_bar, cons_phase, a.status);  // scratch and flag are free again
-            if (!ok) break;
+            if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;  // scratch and flag are free again
 #pragma unroll
             for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -566,6 +624,11 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
                     for (int c = 0; c < 4; ++c) acc[r][nt][c] = 0.f;
             first_ks = -1;
         }
+        return true;
+    };
+    for (int i = 0; i < nsteps; i += 2) {
+        if (!do_step(i, sz_a, sz_b)) break;
+        if (i + 1 < nsteps && !do_step(i + 1, sz_b, sz_a)) break;
     }
 }
 
@@ -586,10 +649,20 @@ int sm_count() {
     return cached[dev];
 }
 
-template <int BITS, int NT, int GS, bool OUT_F32>
+// Programmatic dependent launch is on unless the environment says DMR_PDL=0.
+bool pdl_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("DMR_PDL");
+        v = (e && e[0] == '0') ? 0 : 1;
+    }
+    return v != 0;
+}
+
+template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
 dmr_status_t launch_stream_t(const CUtensorMap &wmap, const StreamArgs &a, int ctas, cudaStream_t st) {
     using Cfg = StreamCfg<BITS, NT, GS>;
-    auto kernel = decode_stream_kernel<BITS, NT, GS, OUT_F32>;
+    auto kernel = decode_stream_kernel<BITS, NT, GS, CE, OUT_F32>;
     static bool configured_on[64] = {};
     bool &configured = configured_on[current_device()];
     if (!configured) {
@@ -609,7 +682,7 @@ dmr_status_t launch_stream_t(const CUtensorMap &wmap, const StreamArgs &a, int c
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, wmap, a);
     if (e != cudaSuccess) {
         g_last_cuda_error = (int)e;
@@ -619,14 +692,14 @@ dmr_status_t launch_stream_t(const CUtensorMap &wmap, const StreamArgs &a, int c
     return check_launch();
 }
 
-template <int BITS, int GS>
+template <int BITS, int GS, bool CE>
 dmr_status_t launch_stream_nt(const CUtensorMap &wmap, const StreamArgs &a, int ctas, dmr_out_t out, cudaStream_t st) {
     if (a.M <= 8) {
-        if (out == DMR_OUT_F32) return launch_stream_t<BITS, 1, GS, true>(wmap, a, ctas, st);
-        return launch_stream_t<BITS, 1, GS, false>(wmap, a, ctas, st);
+        if (out == DMR_OUT_F32) return launch_stream_t<BITS, 1, GS, CE, true>(wmap, a, ctas, st);
+        return launch_stream_t<BITS, 1, GS, CE, false>(wmap, a, ctas, st);
     }
-    if (out == DMR_OUT_F32) return launch_stream_t<BITS, 2, GS, true>(wmap, a, ctas, st);
-    return launch_stream_t<BITS, 2, GS, false>(wmap, a, ctas, st);
+    if (out == DMR_OUT_F32) return launch_stream_t<BITS, 2, GS, CE, true>(wmap, a, ctas, st);
+    return launch_stream_t<BITS, 2, GS, CE, false>(wmap, a, ctas, st);
 }
 
 }  // namespace
@@ -665,6 +738,9 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     a.N = N;
     a.K = K;
     a.g_size = bits == 16 ? K : g;
+    a.g_shift = -1;
+    for (int sh = 0; sh < 31; ++sh)
+        if ((1 << sh) == a.g_size) a.g_shift = sh;
     a.steps_per_group = (K + step_k - 1) / step_k;
     const long long total = (long long)groups * a.steps_per_group;
     if (total > 0x7FFFFFFF) return DMR_ERR_UNSUPPORTED;
@@ -677,10 +753,14 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     if (!make_tensor_map_2d(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, weights, (uint64_t)N, row_bytes, row_bytes, kTileRows,
                             128, TmaSwizzle::k128B))
         return DMR_ERR_CUDA;
-    if (bits == 16) return launch_stream_nt<16, 1>(wmap, a, ctas, out, st);
-    if (bits == 8) return launch_stream_nt<8, 1>(wmap, a, ctas, out, st);
-    if (g == 64) return launch_stream_nt<4, 2>(wmap, a, ctas, out, st);
-    return launch_stream_nt<4, 1>(wmap, a, ctas, out, st);
+    if (bits == 16) return launch_stream_nt<16, 1, false>(wmap, a, ctas, out, st);
+    if (bits == 8) {
+        if (g == 64) return launch_stream_nt<8, 1, true>(wmap, a, ctas, out, st);
+        return launch_stream_nt<8, 1, false>(wmap, a, ctas, out, st);
+    }
+    if (g == 64) return launch_stream_nt<4, 2, true>(wmap, a, ctas, out, st);
+    if (g == 128) return launch_stream_nt<4, 1, true>(wmap, a, ctas, out, st);
+    return launch_stream_nt<4, 1, false>(wmap, a, ctas, out, st);
 }
 
 }  // namespace dmr
