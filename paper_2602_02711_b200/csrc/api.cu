@@ -23,6 +23,7 @@ struct Scratch {
     uint16_t *xg_low = nullptr, *xg_high = nullptr;
     float *partial = nullptr;
     void *stream_scratch = nullptr;  // counters + partial sums of the streaming decode kernel
+    uint16_t *xg_stream = nullptr;   // routed, decode path: 16 gathered activation rows
     size_t bytes = 0;
 };
 
@@ -67,6 +68,10 @@ Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f
     if (low_stream || dense_stream) {
         s.stream_scratch = base + off;
         off += round_up(stream_scratch_bytes(N), 256);
+        if (op == DMR_OP_ROUTED_LINEAR) {
+            s.xg_stream = reinterpret_cast<uint16_t *>(base + off);
+            off += round_up((size_t)16 * K * 2, 256);
+        }
     }
     s.bytes = round_up(off, 256);
     return s;
@@ -91,7 +96,7 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
     if (use_gemm(M, N, K, f.bits, g)) {
         const uint16_t *Xin = X;
         if (sel.idx) {
-            dmr_status_t r = launch_gather_rows(X, K, M, sel.idx, sel.count, ws.xg_low, st);
+            dmr_status_t r = launch_gather_rows(X, K, M, sel.idx, sel.count, 0, ws.xg_low, st);
             if (r != DMR_OK) return r;
             Xin = ws.xg_low;
         }
@@ -111,6 +116,11 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
             Xc = X + (size_t)m0 * K;
             Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
         }
+        if (sel.idx) {  // the kernel reads consecutive rows: gather this chunk's rows first
+            dmr_status_t rg = launch_gather_rows(X, K, mc, s.idx, s.count, s.offset, ws.xg_stream, st);
+            if (rg != DMR_OK) return rg;
+            Xc = ws.xg_stream;
+        }
         dmr_status_t r = launch_stream(Xc, mc, s, qweight, scales, zeros, N, K, f.bits, g, Yc, out, ws.stream_scratch,
                                        ws.status, st);
         if (r != DMR_OK) return r;
@@ -124,7 +134,7 @@ dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, 
     if (use_gemm(M, N, K, 0, K)) {
         const uint16_t *Xin = X;
         if (sel.idx) {
-            dmr_status_t r = launch_gather_rows(X, K, M, sel.idx, sel.count, ws.xg_high, st);
+            dmr_status_t r = launch_gather_rows(X, K, M, sel.idx, sel.count, 0, ws.xg_high, st);
             if (r != DMR_OK) return r;
             Xin = ws.xg_high;
         }
@@ -142,6 +152,11 @@ dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, 
         } else {
             Xc = X + (size_t)m0 * K;
             Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
+        }
+        if (sel.idx) {
+            dmr_status_t rg = launch_gather_rows(X, K, mc, s.idx, s.count, s.offset, ws.xg_stream, st);
+            if (rg != DMR_OK) return rg;
+            Xc = ws.xg_stream;
         }
         dmr_status_t r = launch_stream(Xc, mc, s, W, nullptr, nullptr, N, K, 16, K, Yc, out, ws.stream_scratch, ws.status, st);
         if (r != DMR_OK) return r;

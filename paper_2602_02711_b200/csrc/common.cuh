@@ -84,8 +84,10 @@ GemmPlan gemm_plan(int M, int N, int K, int bits);
 dmr_status_t launch_gemm(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,
                          const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
                          float *partial, int32_t *status, cudaStream_t st);
+// Xg[s] = X[idx[s]] for the list slots coff <= coff + s < *count (s < Mcap); other slots are zero-filled.
+// `idx` is already advanced to slot coff.
 dmr_status_t launch_gather_rows(const uint16_t *X, int K, int Mcap, const int32_t *idx, const int32_t *count,
-                                uint16_t *Xg, cudaStream_t st);
+                                int coff, uint16_t *Xg, cudaStream_t st);
 
 // Any-shape fallback (CUDA cores, one warp per output feature).
 dmr_status_t launch_simple_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight,

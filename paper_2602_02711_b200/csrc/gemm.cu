@@ -347,8 +347,8 @@ splitk_reduce_kernel(const float *__restrict__ partial, int splits, int M, int N
 // are zero-filled so that the tensor core never sees uninitialised memory.
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint16_t *__restrict__ X, int K, int Mcap, const int32_t *__restrict__ idx,
-                   const int32_t *__restrict__ count, uint16_t *__restrict__ Xg) {
-    const int rows = min(*count, Mcap);
+                   const int32_t *__restrict__ count, int coff, uint16_t *__restrict__ Xg) {
+    const int rows = min(*count - coff, Mcap);
     const int vec_per_row = K / 8;
     const size_t total = (size_t)Mcap * vec_per_row;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
@@ -467,11 +467,11 @@ dmr_status_t launch_gemm(const uint16_t *X, int M, RowSel sel, const void *weigh
 }
 
 dmr_status_t launch_gather_rows(const uint16_t *X, int K, int Mcap, const int32_t *idx, const int32_t *count,
-                                uint16_t *Xg, cudaStream_t st) {
+                                int coff, uint16_t *Xg, cudaStream_t st) {
     const size_t total = (size_t)Mcap * (K / 8);
     int blocks = (int)((total + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
-    gather_rows_kernel<<<blocks, 256, 0, st>>>(X, K, Mcap, idx, count, Xg);
+    gather_rows_kernel<<<blocks, 256, 0, st>>>(X, K, Mcap, idx, count, coff, Xg);
     return check_launch();
 }
 

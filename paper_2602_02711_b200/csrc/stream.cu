@@ -12,10 +12,9 @@
 // summation order of an output depends on (N, K) and the SM count only - never on M, on the
 // row's position in the batch or on the other rows.
 //
-// Inside a CTA one producer warp keeps a ring of stages full: the weight box by TMA
-// (cp.async.bulk.tensor, 128-byte swizzle) and the matching activation slice by 16-byte
-// cp.async (which also gathers the rows of a routed batch), both completing on the stage's
-// mbarrier.  Eight consumer warps each own 32 features and one half of the step's k range; the
+// Inside a CTA one producer lane keeps a ring of stages full by TMA (cp.async.bulk.tensor,
+// 128-byte swizzle): the weight box and the matching activation boxes, all completing on the
+// stage's mbarrier (a routed batch is gathered into consecutive rows beforehand).  Eight consumer warps each own 32 features and one half of the step's k range; the
 // product runs on the tensor cores with the weights as the 16-row operand of mma.m16n8k16 and up
 // to 8 (or 2 x 8) activation rows as the 8-column operand.  4-bit codes are unpacked with one
 // LOP3 per two codes ((w >> 4p) & 0x000F000F | 0x43004300 = {128 + q_p, 128 + q_{p+4}} as two
@@ -37,7 +36,7 @@ namespace dmr {
 
 namespace {
 
-constexpr int kR = 1;                                        // 16-feature tiles per consumer warp
+constexpr int kR = 2;                                        // 16-feature tiles per consumer warp
 constexpr int kRowBlocks = 128 / (16 * kR);                  // consumer warps side by side over the features
 constexpr int kConsumerWarps = 2 * kRowBlocks;               // two k halves
 constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
@@ -104,18 +103,6 @@ __device__ __forceinline__ uint2 lds64(uint32_t addr) {
     return v;
 }
 
-// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-
-// One arrival on `bar` once every cp.async issued so far by this thread has landed.
-__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
-
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -129,23 +116,23 @@ template <int BITS>
 struct StepGeom {
     static constexpr int STEP_K = 1024 / BITS;         // weights per 128-byte row: 256, 128, 64
     static constexpr int UNIT_K = STEP_K / 2;          // per k-half warp: 128, 64, 32
-    static constexpr int X_ROW_BYTES = STEP_K * 2;     // activation bytes per row per step
-    static constexpr int X_CHUNKS = X_ROW_BYTES / 16;  // 32, 16, 8
+    static constexpr int X_BOXES = STEP_K / 64;        // activation boxes of 64 k (128 bytes per row): 4, 2, 1
 };
 
-// Where 16-byte chunk c of activation row `slot` sits inside that row of a stage.  Lane (g, t) reads
-// consecutive chunks of row g starting at (its k half) * X_CHUNKS / 2 + t * (chunks per lane); the
-// permutation makes the eight lanes of a shared-memory phase (two rows, four values of t) hit
-// eight different bank groups.
-template <int BITS>
-__device__ __forceinline__ int x_chunk_pos(int c, int slot) {
-    if (BITS == 4) return c ^ (((c >> 3) & 1) << 1) ^ (slot & 1);
-    if (BITS == 8) return c ^ (slot & 1);
-    return c ^ ((slot & 1) << 2);
+// Activation boxes of a stage sit 2304 bytes apart: 2048 for 16 rows of 128 bytes plus 256, so that
+// consecutive boxes start two rows further into the 128-byte swizzle pattern (the pattern is tied to
+// the shared-memory address, chunk ^= (address / 128) % 8).  Lanes t and t + 2 of a warp read the same
+// chunk index of consecutive boxes; the shift sends them to different banks.
+constexpr int kXBoxPitch = 2304;
+
+// Byte offset, inside a stage's activation area, of 16-byte chunk c (k = 8 c .. 8 c + 7 of the step)
+// of batch slot `slot`.
+__device__ __forceinline__ uint32_t x_chunk_offset(int c, int slot) {
+    const int sb = c >> 3, cc = c & 7;
+    return (uint32_t)(sb * kXBoxPitch + slot * 128 + ((cc ^ ((slot + 2 * sb) & 7)) << 4));
 }
 
 struct StreamArgs {
-    const uint16_t *X;        // [*][K] bf16
     const int32_t *idx;       // routed: row of X / Y for batch slot s (nullptr = identity)
     const int32_t *count;     // routed: valid slots in the list (nullptr = M)
     const uint16_t *scales;   // low-bit only
@@ -177,7 +164,8 @@ template <int BITS, int NT, int GS>
 struct StreamCfg {
     using G = StepGeom<BITS>;
     static constexpr int SLOTS = NT * 8;
-    static constexpr int X_STAGE = SLOTS * G::X_ROW_BYTES;
+    static constexpr int X_STAGE = ((G::X_BOXES * kXBoxPitch + 1023) / 1024) * 1024;
+    static constexpr int X_TX = G::X_BOXES * SLOTS * 128;  // bytes the activation boxes deliver
     static constexpr int STAGE = kStepBytes + X_STAGE;
     static constexpr int D_RAW = (kStageBudget * 1024) / STAGE;
     static constexpr int D = D_RAW > kMaxStages ? kMaxStages : D_RAW;
@@ -191,7 +179,8 @@ struct StreamCfg {
 // CE: every unit a warp consumes ends its quantization group (group size == unit size).
 template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
 __global__ void __launch_bounds__(kStreamThreads, 1)
-decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs a) {
+decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ CUtensorMap xmap,
+                     const StreamArgs a) {
     using Cfg = StreamCfg<BITS, NT, GS>;
     using Geo = StepGeom<BITS>;
     constexpr int D = Cfg::D, SLOTS = Cfg::SLOTS, R = kR;
@@ -223,83 +212,56 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
 
     if (threadIdx.x == 0) {
         for (int d = 0; d < D; ++d) {
-            mbar_init(full_bar(d), 1 + 32);
+            mbar_init(full_bar(d), 1);
             mbar_init(empty_bar(d), kConsumerWarps);
         }
         mbar_init(cons_bar, kConsumerWarps);
         fence_barrier_init();
         prefetch_tensor_map(&wmap);
+        prefetch_tensor_map(&xmap);
     }
     __syncthreads();
     pdl_launch_dependents();
 
     if (warp == kConsumerWarps) {
-        // ======================= producer warp =======================
-        // Weights never depend on the preceding kernel: start them before waiting for it
-        // (a routed call must first learn whether it has any row at all).
+        // ======================= producer warp (one lane issues every copy) =======================
+        // Weights never depend on the preceding kernel: start them before waiting for it (a routed
+        // call must first learn whether it has any row at all).  The stage's barrier gets its one
+        // arrival only when the activations are issued, so it cannot complete on weights alone.
         int npre = 0;
-        if (a.count == nullptr && lane == 0) {
-            int rg = rg_first, ks = ks_first;
-            for (; npre < D && npre < nsteps; ++npre) {
-                mbar_expect_tx(full_bar(npre), kStepBytes);
-                tma_load_2d(w_stage(npre), &wmap, full_bar(npre), ks * 128, rg * kTileRows);
+        if (lane == 0) {
+            if (a.count == nullptr) {
+                int rg = rg_first, ks = ks_first;
+                for (; npre < D && npre < nsteps; ++npre) {
+                    mbar_expect_tx_only(full_bar(npre), kStepBytes);
+                    tma_load_2d(w_stage(npre), &wmap, full_bar(npre), ks * 128, rg * kTileRows);
+                    if (++ks == SPG) {
+                        ks = 0;
+                        ++rg;
+                    }
+                }
+            }
+            pdl_wait();
+            const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
+            if (rows <= 0) return;
+            int rg = rg_first, ks = ks_first - 1;
+            for (int i = 0; i < nsteps; ++i) {
+                const int d = i % D;
                 if (++ks == SPG) {
                     ks = 0;
                     ++rg;
                 }
-            }
-        }
-        npre = __shfl_sync(0xFFFFFFFFu, npre, 0);
-        pdl_wait();
-        const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
-        if (rows <= 0) return;
-        // batch slot -> row of X (lane l holds slot l)
-        int my_row = -1;
-        if (lane < SLOTS && lane < rows) my_row = a.idx ? a.idx[lane] : lane;
-        int last_pf_group = -1, last_pf_rg = -1;
-        const int xchunks = rows * Geo::X_CHUNKS;  // slots past `rows` feed output columns nobody reads
-        int rg = rg_first, ks = ks_first - 1;
-        for (int i = 0; i < nsteps; ++i) {
-            const int d = i % D;
-            if (++ks == SPG) {
-                ks = 0;
-                ++rg;
-            }
-            if (i >= D && !mbar_wait(empty_bar(d), (uint32_t)(((i / D) - 1) & 1), a.status)) break;
-            if (i >= npre && lane == 0) {
-                mbar_expect_tx(full_bar(d), kStepBytes);
-                tma_load_2d(w_stage(d), &wmap, full_bar(d), ks * 128, rg * kTileRows);
-            }
-            // activations of this k range, all batch slots
-            const uint32_t xs = x_stage(d);
-            for (int c0 = 0; c0 < xchunks; c0 += 32) {
-                const int ch = c0 + lane;
-                const int slot = ch / Geo::X_CHUNKS, cc = ch % Geo::X_CHUNKS;
-                const int row = __shfl_sync(0xFFFFFFFFu, my_row, slot & 31);
-                const int k = ks * Geo::STEP_K + cc * 8;
-                if (ch < xchunks) {
-                    const bool valid = k < a.K;  // past the end of a ragged row: zeros
-                    const uint16_t *src = valid ? a.X + (size_t)row * a.K + k : a.X;
-                    cp_async16(xs + slot * Geo::X_ROW_BYTES + x_chunk_pos<BITS>(cc, slot) * 16, src, valid ? 16u : 0u);
+                if (i >= D && !mbar_wait(empty_bar(d), (uint32_t)(((i / D) - 1) & 1), a.status)) break;
+                if (i >= npre) {
+                    mbar_expect_tx(full_bar(d), kStepBytes + Cfg::X_TX);
+                    tma_load_2d(w_stage(d), &wmap, full_bar(d), ks * 128, rg * kTileRows);
+                } else {
+                    mbar_expect_tx(full_bar(d), Cfg::X_TX);
                 }
-            }
-            cp_async_arrive(full_bar(d));
-            if (LOWBIT) {
-                // pull the scale / zero sectors of the groups ahead into L2 before the consumers ask
-                const int g0 = group_of_k(ks * Geo::STEP_K);
-                if (rg != last_pf_rg || g0 >= last_pf_group + 16) {
-                    last_pf_rg = rg;
-                    last_pf_group = g0;
-                    const int g1 = min(G - 1, g0 + 15);
+                // activations of this k range: one [slots x 64] box per 64 k, rows past M read as zero
 #pragma unroll
-                    for (int q = 0; q < kTileRows / 32; ++q) {
-                        const int n = min(rg * kTileRows + q * 32 + lane, a.N - 1);
-                        prefetch_l2(a.scales + (size_t)n * G + g0);
-                        prefetch_l2(a.scales + (size_t)n * G + g1);
-                        prefetch_l2(a.zeros + (size_t)n * G + g0);
-                        prefetch_l2(a.zeros + (size_t)n * G + g1);
-                    }
-                }
+                for (int sb = 0; sb < Geo::X_BOXES; ++sb)
+                    tma_load_2d(x_stage(d) + sb * kXBoxPitch, &xmap, full_bar(d), ks * Geo::STEP_K + sb * 64, 0);
             }
         }
         return;
@@ -341,7 +303,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const StreamArgs 
                 if (BITS == 4) c = GS == 1 ? kh * 16 + t * 4 + i4 : kh * 16 + sg * 8 + t * 2 + i4;
                 else if (BITS == 8) c = kh * 8 + t * 2 + i4;
                 else c = kh * 4 + t;
-                x_off[nt][sg][i4] = (uint32_t)((nt * 8 + g) * Geo::X_ROW_BYTES + x_chunk_pos<BITS>(c, g) * 16);
+                x_off[nt][sg][i4] = x_chunk_offset(c, nt * 8 + g);
             }
 
     float acc[R][NT][4], accg[R][NT][4];
@@ -660,7 +622,8 @@ bool pdl_enabled() {
 }
 
 template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
-dmr_status_t launch_stream_t(const CUtensorMap &wmap, const StreamArgs &a, int ctas, cudaStream_t st) {
+dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, const StreamArgs &a, int ctas,
+                             cudaStream_t st) {
     using Cfg = StreamCfg<BITS, NT, GS>;
     auto kernel = decode_stream_kernel<BITS, NT, GS, CE, OUT_F32>;
     static bool configured_on[64] = {};
@@ -683,7 +646,7 @@ dmr_status_t launch_stream_t(const CUtensorMap &wmap, const StreamArgs &a, int c
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, wmap, a);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, wmap, xmap, a);
     if (e != cudaSuccess) {
         g_last_cuda_error = (int)e;
         (void)cudaGetLastError();
@@ -693,13 +656,14 @@ dmr_status_t launch_stream_t(const CUtensorMap &wmap, const StreamArgs &a, int c
 }
 
 template <int BITS, int GS, bool CE>
-dmr_status_t launch_stream_nt(const CUtensorMap &wmap, const StreamArgs &a, int ctas, dmr_out_t out, cudaStream_t st) {
+dmr_status_t launch_stream_nt(const CUtensorMap &wmap, const CUtensorMap &xmap, const StreamArgs &a, int ctas,
+                              dmr_out_t out, cudaStream_t st) {
     if (a.M <= 8) {
-        if (out == DMR_OUT_F32) return launch_stream_t<BITS, 1, GS, CE, true>(wmap, a, ctas, st);
-        return launch_stream_t<BITS, 1, GS, CE, false>(wmap, a, ctas, st);
+        if (out == DMR_OUT_F32) return launch_stream_t<BITS, 1, GS, CE, true>(wmap, xmap, a, ctas, st);
+        return launch_stream_t<BITS, 1, GS, CE, false>(wmap, xmap, a, ctas, st);
     }
-    if (out == DMR_OUT_F32) return launch_stream_t<BITS, 2, GS, CE, true>(wmap, a, ctas, st);
-    return launch_stream_t<BITS, 2, GS, CE, false>(wmap, a, ctas, st);
+    if (out == DMR_OUT_F32) return launch_stream_t<BITS, 2, GS, CE, true>(wmap, xmap, a, ctas, st);
+    return launch_stream_t<BITS, 2, GS, CE, false>(wmap, xmap, a, ctas, st);
 }
 
 }  // namespace
@@ -723,7 +687,6 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
                            void *scratch, int32_t *status, cudaStream_t st) {
     const int step_k = 1024 / bits;
     StreamArgs a;
-    a.X = X;
     a.idx = sel.idx;
     a.count = sel.count;
     a.scales = scales;
@@ -753,14 +716,19 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     if (!make_tensor_map_2d(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, weights, (uint64_t)N, row_bytes, row_bytes, kTileRows,
                             128, TmaSwizzle::k128B))
         return DMR_ERR_CUDA;
-    if (bits == 16) return launch_stream_nt<16, 1, false>(wmap, a, ctas, out, st);
+    // X holds M consecutive rows (for a routed call: the gathered rows); box = [8 or 16 slots][64 k]
+    CUtensorMap xmap;
+    if (!make_tensor_map_2d(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)K * 2,
+                            M <= 8 ? 8 : 16, 64, TmaSwizzle::k128B))
+        return DMR_ERR_CUDA;
+    if (bits == 16) return launch_stream_nt<16, 1, false>(wmap, xmap, a, ctas, out, st);
     if (bits == 8) {
-        if (g == 64) return launch_stream_nt<8, 1, true>(wmap, a, ctas, out, st);
-        return launch_stream_nt<8, 1, false>(wmap, a, ctas, out, st);
+        if (g == 64) return launch_stream_nt<8, 1, true>(wmap, xmap, a, ctas, out, st);
+        return launch_stream_nt<8, 1, false>(wmap, xmap, a, ctas, out, st);
     }
-    if (g == 64) return launch_stream_nt<4, 2, true>(wmap, a, ctas, out, st);
-    if (g == 128) return launch_stream_nt<4, 1, true>(wmap, a, ctas, out, st);
-    return launch_stream_nt<4, 1, false>(wmap, a, ctas, out, st);
+    if (g == 64) return launch_stream_nt<4, 2, true>(wmap, xmap, a, ctas, out, st);
+    if (g == 128) return launch_stream_nt<4, 1, true>(wmap, xmap, a, ctas, out, st);
+    return launch_stream_nt<4, 1, false>(wmap, xmap, a, ctas, out, st);
 }
 
 }  // namespace dmr
