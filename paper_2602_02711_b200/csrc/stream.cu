@@ -170,7 +170,9 @@ struct StreamCfg {
     static constexpr int D_RAW = (kStageBudget * 1024) / STAGE;
     static constexpr int D = D_RAW > kMaxStages ? kMaxStages : D_RAW;
     static constexpr int SCRATCH = SLOTS * kTileRows * 4;
-    static constexpr int BAR_OFF = D * STAGE + SCRATCH;
+    static constexpr int SZ_OFF = D * STAGE + SCRATCH;
+    static constexpr int SZ_WARP = 2 * 16 * kR * GS * 4;  // per consumer warp: two slots of (scale, zero) entries
+    static constexpr int BAR_OFF = SZ_OFF + kConsumerWarps * SZ_WARP;
     static constexpr size_t SMEM = (size_t)BAR_OFF + 512 + 1024 /*alignment slack*/;
 };
 
@@ -314,40 +316,78 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[r][nt][c] = accg[r][nt][c] = 0.f;
 
-    // scale / zero of (feature, group), loaded one step ahead into one of two register sets
-    typedef uint32_t SzRegs[R][2][GS][2];
-    SzRegs sz_a, sz_b;
-    auto load_sz = [&](int rg, int ks, SzRegs &dst) {
+    // Scale and zero point of (feature, group).  Each warp keeps the entries of its own 16R features
+    // for the current and the next step in a private shared-memory area: lane l fetches feature l's
+    // pair two steps ahead (registers `pend`), packs it as scale << 16 | zero (4-bit: | 0x4300, the
+    // bf16 of 128 + zero) one step ahead and every lane then reads the entries of its fragment rows.
+    const uint32_t sz_base = base + Cfg::SZ_OFF + (uint32_t)warp * Cfg::SZ_WARP;
+    auto sz_fetch = [&](int rg_, int ks_, uint32_t (&dst)[GS][2]) {
         if (!LOWBIT) return;
-        const int k0 = ks * Geo::STEP_K + kh * Geo::UNIT_K;
+        const int n = min(rg_ * kTileRows + rb * 16 * R + lane, N - 1);
+        const int k0 = ks_ * Geo::STEP_K + kh * Geo::UNIT_K;
 #pragma unroll
-        for (int r = 0; r < R; ++r)
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int n = min(rg * kTileRows + rb * 16 * R + r * 16 + trow + 8 * h, N - 1);
-#pragma unroll
-                for (int sg = 0; sg < GS; ++sg) {
-                    const int grp = min(group_of_k(k0 + sg * (Geo::UNIT_K / GS)), G - 1);
-                    dst[r][h][sg][0] = __ldg(a.scales + (size_t)n * G + grp);
-                    dst[r][h][sg][1] = __ldg(a.zeros + (size_t)n * G + grp);
-                }
-            }
+        for (int sg = 0; sg < GS; ++sg) {
+            const int grp = min(group_of_k(k0 + sg * (Geo::UNIT_K / GS)), G - 1);
+            dst[sg][0] = __ldg(a.scales + (size_t)n * G + grp);
+            dst[sg][1] = __ldg(a.zeros + (size_t)n * G + grp);
+        }
     };
-    if (nsteps > 0) load_sz(rg_first, ks_first, sz_a);
+    auto sz_store = [&](int slot, const uint32_t (&src)[GS][2]) {
+        if (!LOWBIT) return;
+#pragma unroll
+        for (int sg = 0; sg < GS; ++sg) {
+            const uint32_t v = (src[sg][0] << 16) | src[sg][1] | (BITS == 4 ? 0x4300u : 0u);
+            asm volatile("st.shared.u32 [%0], %1;" ::"r"(sz_base + (uint32_t)(((slot * GS + sg) * 16 * R + lane) * 4)), "r"(v) : "memory");
+        }
+        __syncwarp();
+    };
+    auto step_after = [&](int &rg_, int &ks_) {
+        if (++ks_ == SPG) {
+            ks_ = 0;
+            ++rg_;
+        }
+    };
+    uint32_t pend[GS][2];
+    int rg_pf = rg_first, ks_pf = ks_first;  // step the next fetch is for
+    if (nsteps > 0) {
+        sz_fetch(rg_pf, ks_pf, pend);
+        sz_store(0, pend);
+        step_after(rg_pf, ks_pf);
+    }
+    if (nsteps > 1) {
+        sz_fetch(rg_pf, ks_pf, pend);
+        step_after(rg_pf, ks_pf);
+    }
 
     uint32_t cons_phase = 0;
     int first_ks = -1;  // k step at which this CTA entered the current feature group
     int rg = rg_first, ks = ks_first - 1;
 
-    // One step of the ring: `cur` holds this step's scales / zeros, `nxt` receives the next step's.
-    auto do_step = [&](int i, SzRegs &cur, SzRegs &nxt) -> bool {
+    auto do_step = [&](int i) -> bool {
         const int d = i % D;
         if (++ks == SPG) {
             ks = 0;
             ++rg;
         }
         if (first_ks < 0) first_ks = ks;
-        if (i + 1 < nsteps) load_sz(ks + 1 == SPG ? rg + 1 : rg, ks + 1 == SPG ? 0 : ks + 1, nxt);
+        uint32_t fresh_sz[GS][2];
+        if (i + 2 < nsteps) {
+            sz_fetch(rg_pf, ks_pf, fresh_sz);
+            step_after(rg_pf, ks_pf);
+        }
+        // this step's entries for the lane's fragment rows
+        uint32_t ent[R][2][GS];
+        if (LOWBIT) {
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int sg = 0; sg < GS; ++sg)
+                        asm volatile("ld.shared.u32 %0, [%1];"
+                                     : "=r"(ent[r][h][sg])
+                                     : "r"(sz_base + (uint32_t)((((i & 1) * GS + sg) * 16 * R + r * 16 + trow + 8 * h) * 4)));
+        }
         if (!mbar_wait(full_bar(d), (uint32_t)((i / D) & 1), a.status)) return false;
         const int k0 = ks * Geo::STEP_K + kh * Geo::UNIT_K;
         if (k0 < K) {  // warp-uniform: the unit may lie past the end of a ragged row
@@ -394,8 +434,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                     for (int r = 0; r < R; ++r)
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const uint32_t zz = 0x4300u | cur[r][h][sg][1];  // bf16 of 128 + zero (exact)
-                            zoff[r][h] = prmt(zz, zz, 0x1010);
+                            zoff[r][h] = prmt(ent[r][h][sg], 0u, 0x1010);  // bf16 of 128 + zero (exact), twice
                         }
 #pragma unroll
                     for (int w = 0; w < WW; ++w)
@@ -436,7 +475,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                             uint32_t av[4];
 #pragma unroll
                             for (int h = 0; h < 2; ++h) {
-                                const float zf = __uint_as_float(0x4B000000u | cur[r][h][sg][1]);  // 2^23 + zero
+                                const float zf = __uint_as_float(0x4B000000u | (ent[r][h][sg] & 0xFFu));  // 2^23 + zero
                                 const uint32_t uu = wq[r][h][w];
                                 float f[4];
 #pragma unroll
@@ -472,8 +511,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                     if (closes) {
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
-                            const float s0 = __uint_as_float(cur[r][0][sg][0] << 16);
-                            const float s1 = __uint_as_float(cur[r][1][sg][0] << 16);
+                            const float s0 = __uint_as_float(ent[r][0][sg] & 0xFFFF0000u);
+                            const float s1 = __uint_as_float(ent[r][1][sg] & 0xFFFF0000u);
 #pragma unroll
                             for (int nt = 0; nt < NT; ++nt) {
                                 acc[r][nt][0] = fmaf(s0, accg[r][nt][0], acc[r][nt][0]);
@@ -492,6 +531,17 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar(d));
+        // pack the next step's scale / zero pairs (fetched one step ago) for the whole warp
+        if (i + 1 < nsteps) {
+            sz_store((i + 1) & 1, pend);
+            if (LOWBIT) {
+#pragma unroll
+                for (int sg = 0; sg < GS; ++sg) {
+                    pend[sg][0] = fresh_sz[sg][0];
+                    pend[sg][1] = fresh_sz[sg][1];
+                }
+            }
+        }
 
         // ---- end of this CTA's part of the feature group: combine and write ----
         if (ks == SPG - 1 || i == nsteps - 1) {
@@ -588,10 +638,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         }
         return true;
     };
-    for (int i = 0; i < nsteps; i += 2) {
-        if (!do_step(i, sz_a, sz_b)) break;
-        if (i + 1 < nsteps && !do_step(i + 1, sz_b, sz_a)) break;
-    }
+    for (int i = 0; i < nsteps; ++i)
+        if (!do_step(i)) break;
 }
 
 int current_device() {
