@@ -63,7 +63,7 @@ dmr_status_t launch_dequantize(const uint32_t *qweight, const uint16_t *scales, 
 // Streaming decode kernel (M <= 16): persistent, one CTA per SM, weights read once.  `bits` is 4 or 8
 // for packed codes and 16 for bf16 weights.  `scratch` holds stream_scratch_bytes(N) bytes that are
 // zero before the first use (the kernel leaves its counters zeroed again).
-constexpr int kMaxStreamCtas = 256;
+constexpr int kMaxStreamCtas = 512;
 size_t stream_scratch_bytes(int N);
 bool stream_supported(int M, int N, int K, int bits, int g);
 dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,

@@ -77,6 +77,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
     return false;
 }
 
+// The same bounded wait for a thread that has nothing to do until the phase completes and shares
+// its scheduler with busy warps: the hardware may suspend it for up to `suspend_ns` per try, and
+// it sleeps between tries instead of spinning, so that it takes almost no issue slots.
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, int32_t *status, uint32_t suspend_ns = 2000) {
+    for (uint32_t i = 0; i < (kWaitLimit >> 4); ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity), "r"(suspend_ns)
+            : "memory");
+        if (ok) return true;
+        __nanosleep(100);
+    }
+    if (status) atomicExch(status, (int32_t)DMR_ERR_TIMEOUT);
+    return false;
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap *map, uint32_t bar, int32_t x,
                                             int32_t y) {
     asm volatile(

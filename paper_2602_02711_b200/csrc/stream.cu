@@ -5,7 +5,7 @@
 //
 // Work decomposition.  The weight matrix is cut into steps of [128 features x 128 bytes] (256
 // 4-bit codes, 128 8-bit codes or 64 bf16 weights per feature).  Steps are numbered feature-group
-// major, k minor, and CTA c of the (at most one per SM) grid takes the contiguous range
+// major, k minor, and CTA c of the persistent grid (one or two CTAs per SM) takes the contiguous range
 // [c * total / ctas, (c + 1) * total / ctas): every SM streams the same number of bytes whatever
 // the shape.  A feature group whose steps are shared by several CTAs is finished by the last of
 // them to arrive, which adds the partial sums in CTA order (no floating-point atomics), so the
@@ -180,7 +180,7 @@ struct StreamCfg {
 // GS: quantization groups per 128-code unit (2 only for 4-bit codes with 64-wide groups).
 // CE: every unit a warp consumes ends its quantization group (group size == unit size).
 template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
-__global__ void __launch_bounds__(kStreamThreads, 1)
+__global__ void __launch_bounds__(kStreamThreads, NT == 1 ? 2 : 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ CUtensorMap xmap,
                      const StreamArgs a) {
     using Cfg = StreamCfg<BITS, NT, GS>;
@@ -211,6 +211,26 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
     // quantization group of input feature k without a division in the common cases
     auto group_of_k = [&](int k) { return a.g_shift >= 0 ? (k >> a.g_shift) : (G == 1 ? 0 : k / a.g_size); };
     const int rg_first = beg / SPG, ks_first = beg - rg_first * SPG;
+    // Order of work.  A range that ends inside a feature group (shared with the next CTA) takes those
+    // last n_tail steps FIRST and then runs from its beginning up to that group: both CTAs of a shared
+    // group then produce their parts early and the fix-up hides behind the rest of the stream, and
+    // every CTA ends on a feature group it owns alone.
+    const int rg_last = (end - 1) / SPG;
+    const int n_tail = (end % SPG != 0 && rg_last > rg_first) ? end - rg_last * SPG : 0;
+    struct Cursor {
+        int rg, ks, i;
+    };
+    auto cursor_start = [&]() { return n_tail > 0 ? Cursor{rg_last, 0, 0} : Cursor{rg_first, ks_first, 0}; };
+    auto cursor_next = [&](Cursor &c) {
+        if (++c.i == n_tail) {
+            c.rg = rg_first;
+            c.ks = ks_first;
+        } else if (++c.ks == SPG) {
+            c.ks = 0;
+            ++c.rg;
+        }
+    };
+    auto end_of_part = [&](int i) { return i == n_tail - 1 || i == nsteps - 1; };
 
     if (threadIdx.x == 0) {
         for (int d = 0; d < D; ++d) {
@@ -233,27 +253,22 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         int npre = 0;
         if (lane == 0) {
             if (a.count == nullptr) {
-                int rg = rg_first, ks = ks_first;
+                Cursor c = cursor_start();
                 for (; npre < D && npre < nsteps; ++npre) {
                     mbar_expect_tx_only(full_bar(npre), kStepBytes);
-                    tma_load_2d(w_stage(npre), &wmap, full_bar(npre), ks * 128, rg * kTileRows);
-                    if (++ks == SPG) {
-                        ks = 0;
-                        ++rg;
-                    }
+                    tma_load_2d(w_stage(npre), &wmap, full_bar(npre), c.ks * 128, c.rg * kTileRows);
+                    cursor_next(c);
                 }
             }
             pdl_wait();
             const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
             if (rows <= 0) return;
-            int rg = rg_first, ks = ks_first - 1;
+            Cursor c = cursor_start();
             for (int i = 0; i < nsteps; ++i) {
                 const int d = i % D;
-                if (++ks == SPG) {
-                    ks = 0;
-                    ++rg;
-                }
-                if (i >= D && !mbar_wait(empty_bar(d), (uint32_t)(((i / D) - 1) & 1), a.status)) break;
+                const int rg = c.rg, ks = c.ks;
+                cursor_next(c);
+                if (i >= D && !mbar_wait_idle(empty_bar(d), (uint32_t)(((i / D) - 1) & 1), a.status)) break;
                 if (i >= npre) {
                     mbar_expect_tx(full_bar(d), kStepBytes + Cfg::X_TX);
                     tma_load_2d(w_stage(d), &wmap, full_bar(d), ks * 128, rg * kTileRows);
@@ -341,39 +356,31 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         }
         __syncwarp();
     };
-    auto step_after = [&](int &rg_, int &ks_) {
-        if (++ks_ == SPG) {
-            ks_ = 0;
-            ++rg_;
-        }
-    };
     uint32_t pend[GS][2];
-    int rg_pf = rg_first, ks_pf = ks_first;  // step the next fetch is for
+    Cursor pf = cursor_start();  // step the next fetch is for
     if (nsteps > 0) {
-        sz_fetch(rg_pf, ks_pf, pend);
+        sz_fetch(pf.rg, pf.ks, pend);
         sz_store(0, pend);
-        step_after(rg_pf, ks_pf);
+        cursor_next(pf);
     }
     if (nsteps > 1) {
-        sz_fetch(rg_pf, ks_pf, pend);
-        step_after(rg_pf, ks_pf);
+        sz_fetch(pf.rg, pf.ks, pend);
+        cursor_next(pf);
     }
 
     uint32_t cons_phase = 0;
     int first_ks = -1;  // k step at which this CTA entered the current feature group
-    int rg = rg_first, ks = ks_first - 1;
+    Cursor cur = cursor_start();
 
     auto do_step = [&](int i) -> bool {
         const int d = i % D;
-        if (++ks == SPG) {
-            ks = 0;
-            ++rg;
-        }
+        const int rg = cur.rg, ks = cur.ks;
+        cursor_next(cur);
         if (first_ks < 0) first_ks = ks;
         uint32_t fresh_sz[GS][2];
         if (i + 2 < nsteps) {
-            sz_fetch(rg_pf, ks_pf, fresh_sz);
-            step_after(rg_pf, ks_pf);
+            sz_fetch(pf.rg, pf.ks, fresh_sz);
+            cursor_next(pf);
         }
         // this step's entries for the lane's fragment rows
         uint32_t ent[R][2][GS];
@@ -507,7 +514,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                     // lies in another group, in another feature group or outside this CTA's range
                     const int kpart = k0 + sg * (Geo::UNIT_K / GS);
                     const bool closes = CE || group_of_k(kpart + Geo::STEP_K) != group_of_k(kpart) || ks == SPG - 1 ||
-                                        i == nsteps - 1 || kpart + Geo::STEP_K >= K;
+                                        end_of_part(i) || kpart + Geo::STEP_K >= K;
                     if (closes) {
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
@@ -544,7 +551,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         }
 
         // ---- end of this CTA's part of the feature group: combine and write ----
-        if (ks == SPG - 1 || i == nsteps - 1) {
+        if (ks == SPG - 1 || end_of_part(i)) {
             const bool complete = first_ks == 0 && ks == SPG - 1;
             // k half 1 parks its sums, k half 0 adds them (fixed order) and parks the total
             if (kh == 1) {
@@ -580,26 +587,35 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
             if (complete) {
                 for (int o = threadIdx.x; o < SLOTS * kTileRows; o += kConsumerWarps * 32) store_y(o, scratch[o]);
             } else {
-                // shared feature group: leave the partial sums in the scratch area; the CTA that
-                // arrives last adds all parts in CTA order and writes the result
+                // Shared feature group: the CTA that arrives last adds all parts in CTA order and writes
+                // the result.  A CTA that finds every other part already published is that CTA and
+                // keeps its own part in shared memory; otherwise it publishes its part and counts in.
                 const int which = beg > rg * SPG ? 0 : 1;
-                float4 *mine = reinterpret_cast<float4 *>(a.partial + ((size_t)cta * 2 + which) * (16 * kTileRows));
-                for (int o4 = threadIdx.x; o4 < SLOTS * kTileRows / 4; o4 += kConsumerWarps * 32)
-                    mine[o4] = reinterpret_cast<const float4 *>(scratch)[o4];
-                __threadfence();
-                if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
                 const long long s_first = (long long)rg * SPG, s_last = s_first + SPG - 1;
                 const int c_first = (int)(((s_first + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
                 const int c_last = (int)(((s_last + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
                 if (threadIdx.x == 0) {
-                    const int old = atomicAdd(a.counters + rg, 1);
-                    const int last = old == c_last - c_first;
-                    if (last) a.counters[rg] = 0;  // leave the counter ready for the next call
-                    __threadfence();
-                    *flag = last;
+                    int seen;
+                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.counters + rg) : "memory");
+                    *flag = seen == c_last - c_first ? 2 : 0;
                 }
                 if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
-                if (*flag) {
+                int role = *flag;  // 2: reduce with the own part still in shared memory
+                if (role == 0) {
+                    float4 *mine = reinterpret_cast<float4 *>(a.partial + ((size_t)cta * 2 + which) * (16 * kTileRows));
+                    for (int o4 = threadIdx.x; o4 < SLOTS * kTileRows / 4; o4 += kConsumerWarps * 32)
+                        mine[o4] = reinterpret_cast<const float4 *>(scratch)[o4];
+                    if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
+                    if (threadIdx.x == 0) {
+                        __threadfence();  // the parts stored by the whole CTA before the barrier become visible first
+                        const int old = atomicAdd(a.counters + rg, 1);
+                        __threadfence();
+                        *flag = old == c_last - c_first ? 1 : 0;
+                    }
+                    if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
+                    role = *flag;  // 1: reduce from the published parts
+                }
+                if (role != 0) {
                     // loads of up to eight parts are in flight together; the additions keep CTA order
                     for (int o4 = threadIdx.x; o4 < SLOTS * kTileRows / 4; o4 += kConsumerWarps * 32) {
                         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -609,7 +625,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                             for (int u = 0; u < 8; ++u) {
                                 const int cj = min(cj0 + u, c_last);
                                 const int wj = range_begin(cj, ctas, a.total_steps) > s_first ? 0 : 1;
-                                p[u] = __ldcg(reinterpret_cast<const float4 *>(a.partial + ((size_t)cj * 2 + wj) * (16 * kTileRows)) + o4);
+                                if (role == 2 && cj == cta) p[u] = reinterpret_cast<const float4 *>(scratch)[o4];
+                                else p[u] = __ldcg(reinterpret_cast<const float4 *>(a.partial + ((size_t)cj * 2 + wj) * (16 * kTileRows)) + o4);
                             }
 #pragma unroll
                             for (int u = 0; u < 8; ++u)
@@ -625,6 +642,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                         store_y(4 * o4 + 2, v.z);
                         store_y(4 * o4 + 3, v.w);
                     }
+                    if (threadIdx.x == 0) a.counters[rg] = 0;  // leave the counter ready for the next call
                 }
             }
             if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;  // scratch and flag are free again
@@ -756,7 +774,7 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     const long long total = (long long)groups * a.steps_per_group;
     if (total > 0x7FFFFFFF) return DMR_ERR_UNSUPPORTED;
     a.total_steps = (int)total;
-    int ctas = sm_count();
+    int ctas = sm_count() * (M <= 8 ? 2 : 1);  // the 8-row kernels fit twice on an SM
     if (ctas > kMaxStreamCtas) ctas = kMaxStreamCtas;
     if (ctas > a.total_steps) ctas = a.total_steps;
     CUtensorMap wmap;
