@@ -100,6 +100,8 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
             if (r != DMR_OK) return r;
             Xin = ws.xg_low;
         }
+        if (prefill_supported(M, N, K, f.bits, g))
+            return launch_prefill(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.status, st);
         return launch_gemm(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.partial, ws.status, st);
     }
     if (!stream_supported(M < 16 ? M : 16, N, K, f.bits, g))

@@ -1,0 +1,382 @@
+// Prefill-sized low-bit linear layers (M in the hundreds and above): a persistent, warp-specialised
+// tcgen05 GEMM with the dequantisation fused into the operand pipeline.  Prefill is a dense
+// contraction (its cost is folded into the per-token latency, App. "Latency coefficients"), so it
+// belongs on the tensor cores.
+//
+// Orientation: the weights are the 128-row operand (D[n][m] = sum_k W^[n][k] X[m][k]), one
+// tensor-memory lane per output feature, BN (128 or 256) activation rows as the N operand.
+//
+// Per 64-wide k block and stage of the ring:
+//   warp 0      TMA: the packed code tile [128 features x 32 or 64 bytes] and the activation tile
+//               [BN rows x 128 bytes, 128-byte swizzle] land in shared memory (one mbarrier);
+//   warps 2..5  one thread per feature row turns its codes into the bf16 weights s * (q - zero)
+//               (exact integer q - zero, then ONE rounding of the product: the nearest bf16 of
+//               the dequantized weight) and stores them as the swizzled K-major A tile;
+//   warp 1      one lane issues four tcgen05.mma (128 x BN x 16) that accumulate into one of two
+//               fp32 accumulators in tensor memory, and commits the stage back to the producer;
+//   warps 6..9  drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
+//               next tile's MMAs run into the other accumulator.
+// CTAs are persistent: CTA b takes tiles b, b + grid, ...  Every wait is bounded.
+#include <cuda_bf16.h>
+
+#include "sm100.cuh"
+
+namespace dmr {
+
+namespace {
+
+constexpr int PM = 128;  // features per tile (MMA M)
+constexpr int PK = 64;   // k per stage
+
+template <int BITS, int BN>
+struct PrefillCfg {
+    static constexpr int A_BYTES = PM * PK * 2;              // 16 KB of bf16 weights
+    static constexpr int B_BYTES = BN * PK * 2;              // activations
+    static constexpr int P_ROW = PK * BITS / 8;              // packed bytes per feature per stage
+    static constexpr int P_BYTES = PM * P_ROW;               // 4 or 8 KB
+    static constexpr int STAGE = A_BYTES + B_BYTES + ((P_BYTES + 1023) / 1024) * 1024;
+    static constexpr int S_RAW = (212 * 1024) / STAGE;
+    static constexpr int S = S_RAW > 8 ? 8 : S_RAW;
+    static constexpr int TMEM_COLS = 2 * BN;                 // two accumulators
+    static constexpr int THREADS = 320;
+    static constexpr size_t SMEM = (size_t)S * STAGE + 1024 /*alignment*/ + 512 /*barriers*/;
+};
+
+struct PrefillArgs {
+    const uint16_t *scales;
+    const uint8_t *zeros;
+    void *Y;
+    const int32_t *idx;    // routed: output row of batch slot m (nullptr = identity)
+    const int32_t *count;  // routed: number of valid slots (nullptr = M)
+    int32_t *status;
+    int M, N, K, g_size;
+    int n_tiles, m_tiles;
+};
+
+__device__ __forceinline__ uint32_t p_lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));
+    return r;
+}
+__device__ __forceinline__ uint32_t p_prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+__device__ __forceinline__ uint32_t p_sub_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t p_mul_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t p_pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+template <int BITS, int BN, bool OUT_F32>
+__global__ void __launch_bounds__(PrefillCfg<BITS, BN>::THREADS, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const PrefillArgs a) {
+    using Cfg = PrefillCfg<BITS, BN>;
+    constexpr int S = Cfg::S;
+    extern __shared__ uint8_t smem_dyn[];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    uint8_t *base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+    auto a_tile = [&](int s) { return base + (uint32_t)s * Cfg::STAGE; };
+    auto b_tile = [&](int s) { return base + (uint32_t)s * Cfg::STAGE + Cfg::A_BYTES; };
+    auto p_tile = [&](int s) { return base + (uint32_t)s * Cfg::STAGE + Cfg::A_BYTES + Cfg::B_BYTES; };
+    const uint32_t bar_base = base + (uint32_t)S * Cfg::STAGE;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 64u + 8u * s; };
+    auto ready_bar = [&](int s) { return bar_base + 128u + 8u * s; };
+    auto tfull_bar = [&](int b) { return bar_base + 192u + 8u * b; };
+    auto tempty_bar = [&](int b) { return bar_base + 208u + 8u * b; };
+    const uint32_t tmem_slot = bar_base + 224u;
+    volatile uint32_t *tmem_slot_ptr = reinterpret_cast<volatile uint32_t *>(base_ptr + S * Cfg::STAGE + 224);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+            mbar_init(ready_bar(s), 4);   // one arrival per unpack warp
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 4);  // one arrival per epilogue warp
+        }
+        fence_barrier_init();
+        prefetch_tensor_map(&map_w);
+        prefetch_tensor_map(&map_x);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    const int nkb = a.K / PK;
+    // a routed call sizes the grid for M rows but only the first `rows` slots hold anything
+    const int rows = a.count ? min(*a.count, a.M) : a.M;
+    const int total_tiles = a.n_tiles * ((rows + BN - 1) / BN);
+    const int G = a.K / a.g_size;
+    const int kb_per_group = a.g_size / PK;  // >= 1
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            constexpr uint32_t TX = Cfg::B_BYTES + Cfg::P_BYTES;
+            uint32_t it = 0;  // k blocks issued so far, over all tiles
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int n0 = (tile % a.n_tiles) * PM, m0 = (tile / a.n_tiles) * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % S;
+                    if (it >= (uint32_t)S && !mbar_wait(empty_bar(s), ((it / S) - 1) & 1, a.status)) {
+                        ok = false;
+                        break;
+                    }
+                    mbar_expect_tx(full_bar(s), TX);
+                    tma_load_2d(b_tile(s), &map_x, full_bar(s), kb * PK, m0);
+                    tma_load_2d(p_tile(s), &map_w, full_bar(s), kb * Cfg::P_ROW, n0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            constexpr uint32_t IDESC = umma_idesc_bf16(PM, BN);
+            uint32_t it = 0, tile_it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+                const int buf = tile_it & 1;
+                // the epilogue must have drained this accumulator (used two tiles ago)
+                if (tile_it >= 2 && !mbar_wait(tempty_bar(buf), ((tile_it >> 1) - 1) & 1, a.status)) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % S;
+                    if (!mbar_wait(ready_bar(s), (it / S) & 1, a.status)) {
+                        ok = false;
+                        break;
+                    }
+                    tcgen05_fence_after();
+#pragma unroll
+                    for (int j = 0; j < PK / 16; ++j)
+                        umma_bf16_ss(d_tmem, umma_desc_sw128(a_tile(s) + j * 32), umma_desc_sw128(b_tile(s) + j * 32), IDESC,
+                                     (kb == 0 && j == 0) ? 0u : 1u);
+                    umma_commit(empty_bar(s));
+                }
+                if (ok) umma_commit(tfull_bar(buf));
+            }
+        }
+    } else if (warp < 6) {
+        // ================= unpack warps: codes -> bf16 weights s * (q - zero) =================
+        const int r = (warp - 2) * 32 + lane;  // feature row of the tile
+        const uint32_t swz = (uint32_t)(r & 7);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int n = min((tile % a.n_tiles) * PM + r, a.N - 1);
+            const uint16_t *sp = a.scales + (size_t)n * G;
+            const uint8_t *zp = a.zeros + (size_t)n * G;
+            uint32_t sb = __ldg(sp), zb = __ldg(zp);
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const int s = it % S;
+                // scale / zero of the next k block's group, fetched while this block is unpacked
+                uint32_t sb_next = sb, zb_next = zb;
+                if (kb + 1 < nkb && (kb + 1) % kb_per_group == 0) {
+                    const int grp = (kb + 1) / kb_per_group;
+                    sb_next = __ldg(sp + grp);
+                    zb_next = __ldg(zp + grp);
+                }
+                if (!mbar_wait(full_bar(s), (it / S) & 1, a.status)) {
+                    ok = false;
+                    break;
+                }
+                const uint32_t src = p_tile(s) + r * Cfg::P_ROW;
+                const uint32_t dst = a_tile(s) + r * 128;
+                if (BITS == 4) {
+                    uint32_t w[8];
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(src));
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(src + 16));
+                    const uint32_t zz = 0x4300u | zb;             // bf16 of 128 + zero
+                    const uint32_t zoff = zz | (zz << 16);
+                    const uint32_t s2 = sb | (sb << 16);          // the bf16 scale twice
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {  // word c = codes 8c .. 8c+7 = 16-byte chunk c of the row
+                        const uint32_t d04 = p_mul_bf16x2(p_sub_bf16x2(p_lop3_and_or(w[c], 0x000F000Fu, 0x43004300u), zoff), s2);
+                        const uint32_t d15 = p_mul_bf16x2(p_sub_bf16x2(p_lop3_and_or(w[c] >> 4, 0x000F000Fu, 0x43004300u), zoff), s2);
+                        const uint32_t d26 = p_mul_bf16x2(p_sub_bf16x2(p_lop3_and_or(w[c] >> 8, 0x000F000Fu, 0x43004300u), zoff), s2);
+                        const uint32_t d37 = p_mul_bf16x2(p_sub_bf16x2(p_lop3_and_or(w[c] >> 12, 0x000F000Fu, 0x43004300u), zoff), s2);
+                        const uint32_t o01 = p_prmt(d04, d15, 0x5410), o45 = p_prmt(d04, d15, 0x7632);
+                        const uint32_t o23 = p_prmt(d26, d37, 0x5410), o67 = p_prmt(d26, d37, 0x7632);
+                        const uint32_t addr = dst + ((((uint32_t)c) ^ swz) << 4);
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(o01), "r"(o23), "r"(o45), "r"(o67) : "memory");
+                    }
+                } else {
+                    const float zf = __uint_as_float(0x4B000000u | zb);  // 2^23 + zero
+                    const float sf = __uint_as_float(sb << 16);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {  // chunk c = codes 8c .. 8c+7 = packed words 2c, 2c+1
+                        uint32_t w0, w1;
+                        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w0), "=r"(w1) : "r"(src + 8 * c));
+                        uint32_t o[4];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t u = h ? w1 : w0;
+                            float f[4];
+#pragma unroll
+                            for (int b = 0; b < 4; ++b)  // (q - zero) exactly, times the scale exactly (8 x 8 bits)
+                                f[b] = __fmul_rn(__fsub_rn(__uint_as_float(p_prmt(u, 0x4B000000u, 0x7650u + (uint32_t)b)), zf), sf);
+                            o[2 * h] = p_pack_bf16x2(f[0], f[1]);  // the one rounding
+                            o[2 * h + 1] = p_pack_bf16x2(f[2], f[3]);
+                        }
+                        const uint32_t addr = dst + ((((uint32_t)c) ^ swz) << 4);
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                    }
+                }
+                fence_proxy_async_smem();  // the tile must be visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(ready_bar(s));
+                sb = sb_next;
+                zb = zb_next;
+            }
+        }
+    } else {
+        // ================= epilogue warps =================
+        const int q = warp & 3;        // tensor-memory lane quadrant this warp may read
+        const int r = q * 32 + lane;   // feature row of the tile
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        uint32_t tile_it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
+            const int buf = tile_it & 1;
+            const int n = (tile % a.n_tiles) * PM + r, m0 = (tile / a.n_tiles) * BN;
+            if (!mbar_wait(tfull_bar(buf), (tile_it >> 1) & 1, a.status)) break;
+            tcgen05_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t u[32];
+                tmem_ld_x16(lane_addr + (uint32_t)(buf * BN + c0), *reinterpret_cast<uint32_t(*)[16]>(&u[0]));
+                tmem_ld_x16(lane_addr + (uint32_t)(buf * BN + c0 + 16), *reinterpret_cast<uint32_t(*)[16]>(&u[16]));
+                tmem_ld_wait();
+                if (c0 + 32 >= BN) {  // everything of this accumulator is in registers: hand it back
+                    tcgen05_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(buf));
+                }
+                if (n < a.N) {
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const int m = m0 + c0 + c;
+                        if (m < rows) {
+                            const int row = a.idx ? a.idx[m] : m;
+                            const float v = __uint_as_float(u[c]);
+                            if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
+                            else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown: every role's loop is bounded, so all warps arrive here ----
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+template <int BITS, int BN>
+dmr_status_t launch_prefill_t(const CUtensorMap &map_w, const CUtensorMap &map_x, const PrefillArgs &a, int grid,
+                              dmr_out_t out, cudaStream_t st) {
+    using Cfg = PrefillCfg<BITS, BN>;
+    auto launch = [&](auto kernel) -> dmr_status_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            return DMR_ERR_CUDA;
+        }
+        kernel<<<grid, Cfg::THREADS, Cfg::SMEM, st>>>(map_w, map_x, a);
+        return check_launch();
+    };
+    if (out == DMR_OUT_F32) return launch(prefill_kernel<BITS, BN, true>);
+    return launch(prefill_kernel<BITS, BN, false>);
+}
+
+int prefill_sm_count() {
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            cached = n;
+        else
+            cached = 148;
+    }
+    return cached;
+}
+
+// Activation rows per tile: 256 halves the unpack work and shared-memory traffic per flop, 128 fills
+// the last wave better when there are few tiles.  Depends on (M, N) only.
+int prefill_bn(int M, int N, int sms) {
+    const int n_tiles = (N + PM - 1) / PM;
+    auto score = [&](int bn, double rate) {
+        const long long t = (long long)n_tiles * ((M + bn - 1) / bn);
+        const long long waves = (t + sms - 1) / sms;
+        return rate * (double)t / (double)(waves * sms);
+    };
+    return score(256, 1.0) >= score(128, 0.8) ? 256 : 128;
+}
+
+}  // namespace
+
+bool prefill_supported(int M, int N, int K, int bits, int g) {
+    (void)N;
+    return M > 128 && (bits == 4 || bits == 8) && K % PK == 0 && g % PK == 0;
+}
+
+dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qweight, const uint16_t *scales,
+                            const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
+                            int32_t *status, cudaStream_t st) {
+    const int sms = prefill_sm_count();
+    const int bn = prefill_bn(M, N, sms);
+    CUtensorMap map_w, map_x;
+    if (!make_tensor_map_2d(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)K * 2,
+                            (uint32_t)bn, PK, TmaSwizzle::k128B))
+        return DMR_ERR_CUDA;
+    const uint64_t row_bytes = (uint64_t)K * bits / 8;
+    if (!make_tensor_map_2d(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qweight, (uint64_t)N, row_bytes, row_bytes, PM,
+                            (uint32_t)(PK * bits / 8), TmaSwizzle::kNone))
+        return DMR_ERR_CUDA;
+    PrefillArgs a;
+    a.scales = scales;
+    a.zeros = zeros;
+    a.Y = Y;
+    a.idx = sel.idx;
+    a.count = sel.count;
+    a.status = status;
+    a.M = M;
+    a.N = N;
+    a.K = K;
+    a.g_size = g;
+    a.n_tiles = (N + PM - 1) / PM;
+    a.m_tiles = (M + bn - 1) / bn;
+    const long long tiles = (long long)a.n_tiles * a.m_tiles;
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    if (bits == 4) return bn == 256 ? launch_prefill_t<4, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<4, 128>(map_w, map_x, a, grid, out, st);
+    return bn == 256 ? launch_prefill_t<8, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<8, 128>(map_w, map_x, a, grid, out, st);
+}
+
+}  // namespace dmr

@@ -252,6 +252,12 @@ def test_routed_linear_int8_and_ragged():
     routed_case(23, 136, 384, 8, 0, mask)
 
 
+def test_routed_linear_prefill_sized_batch():
+    # above 128 rows both the routed and the unrouted call take the persistent tensor-core kernel
+    mask = inputs.precision_mask(300, 0.3, seed=15)
+    routed_case(300, 264, 512, 4, 128, mask)
+
+
 def test_routed_permutation_equivariance():
     M, N, K = 16, 264, 512
     mask = inputs.precision_mask(M, 0.4, seed=13)
