@@ -225,9 +225,9 @@ dmr_status_t dmr_lowbit_linear(const void *X_bf16, int M, const void *qweight, c
     if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
     if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
     if (!aligned16(qweight)) return DMR_ERR_ALIGNMENT;
+    if (M == 0) return DMR_OK;  // nothing to do, no workspace needed
     if (!workspace || workspace_bytes < dmr_workspace_bytes(DMR_OP_LOWBIT_LINEAR, M, N, K, f)) return DMR_ERR_WORKSPACE;
     if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
-    if (M == 0) return DMR_OK;
     RowSel sel = {nullptr, nullptr, 0};
     const Scratch ws = carve(workspace, DMR_OP_LOWBIT_LINEAR, M, N, K, f);
     return run_lowbit(reinterpret_cast<const uint16_t *>(X_bf16), M, sel, reinterpret_cast<const uint32_t *>(qweight),
@@ -242,9 +242,9 @@ dmr_status_t dmr_dense_linear(const void *X_bf16, int M, const void *W_bf16, int
     if (!W_bf16) return DMR_ERR_INVALID_ARG;
     if (!aligned16(W_bf16)) return DMR_ERR_ALIGNMENT;
     dmr_qformat_t f = {4, 0};
+    if (M == 0) return DMR_OK;  // nothing to do, no workspace needed
     if (!workspace || workspace_bytes < dmr_workspace_bytes(DMR_OP_DENSE_LINEAR, M, N, K, f)) return DMR_ERR_WORKSPACE;
     if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
-    if (M == 0) return DMR_OK;
     RowSel sel = {nullptr, nullptr, 0};
     const Scratch ws = carve(workspace, DMR_OP_DENSE_LINEAR, M, N, K, f);
     return run_dense(reinterpret_cast<const uint16_t *>(X_bf16), M, sel, reinterpret_cast<const uint16_t *>(W_bf16), N,
@@ -269,9 +269,9 @@ dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, c
     if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
     if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
     if (!aligned16(W_bf16) || !aligned16(qweight)) return DMR_ERR_ALIGNMENT;
+    if (M == 0) return DMR_OK;  // nothing to do, no workspace needed
     if (!workspace || workspace_bytes < dmr_workspace_bytes(DMR_OP_ROUTED_LINEAR, M, N, K, f)) return DMR_ERR_WORKSPACE;
     if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
-    if (M == 0) return DMR_OK;
     cudaStream_t st = (cudaStream_t)stream;
     const Scratch ws = carve(workspace, DMR_OP_ROUTED_LINEAR, M, N, K, f);
     r = launch_route_partition(mask, M, ws.idx_high, ws.idx_low, ws.counts, st);
