@@ -142,6 +142,28 @@ dmr_status_t dmr_lowbit_linear_host(const void *X_host, int M, const void *qweig
                                     size_t staging_bytes, void *workspace, size_t workspace_bytes,
                                     void *stream);
 
+/*
+ * No counterpart in the paper: a variant of dmr_lowbit_linear (M <= 16, the decode kernel) for
+ * callers that cannot allocate device memory when they call - for example a serving loop that
+ * gave all free memory to its cache pool at start-up, or code running inside another program's
+ * step that must not touch its allocator (cudaMalloc can also stall the whole device).  It takes
+ * no workspace: the kernel's scratch (counters, partial sums, a status word; about 8.5 MB) is a
+ * fixed array inside the library, which every GPU that loads the library holds until exit.
+ *   - Limits: 1 <= M <= 16, N <= dmr_noalloc_max_n() (65536), formats the decode kernel takes
+ *     (4-bit with group 64 or a multiple of 128, 8-bit with a multiple of 64); anything else
+ *     returns DMR_ERR_UNSUPPORTED and launches nothing.  X, qweight, scales, zeros and Y are the
+ *     caller's device buffers exactly as for dmr_lowbit_linear; the result is identical to it.
+ *   - The first call on each device looks up the array's device address (no allocation); make
+ *     that first call with the device current and before any stream capture begins.
+ *   - The call allocates and frees nothing.  It clears the status word itself; all calls on one
+ *     device share the one array, so two calls that may run on the GPU at the same time (two
+ *     streams, two threads) race - serialise them or use dmr_lowbit_linear with workspaces.
+ */
+int dmr_noalloc_max_n(void);
+dmr_status_t dmr_lowbit_linear_noalloc(const void *X_bf16, int M, const void *qweight, const void *scales,
+                                       const void *zeros, int N, int K, dmr_qformat_t f, void *Y,
+                                       dmr_out_t out, void *stream);
+
 /* Reads the status word a previous call may have set in `workspace` (DMR_OK or DMR_ERR_TIMEOUT).
  * Synchronises `stream`. */
 dmr_status_t dmr_workspace_status(const void *workspace, void *stream);

@@ -71,6 +71,9 @@ def lib() -> ctypes.CDLL:
     L.dmr_host_staging_bytes.argtypes = [i32, i32, i32, i32]
     L.dmr_lowbit_linear_host.restype = i32
     L.dmr_lowbit_linear_host.argtypes = [vp, i32, vp, vp, vp, i32, i32, QFormat, vp, i32, vp, sz, vp, sz, vp]
+    L.dmr_noalloc_max_n.restype = i32
+    L.dmr_lowbit_linear_noalloc.restype = i32
+    L.dmr_lowbit_linear_noalloc.argtypes = [vp, i32, vp, vp, vp, i32, i32, QFormat, vp, i32, vp]
     L.dmr_workspace_status.restype = i32
     L.dmr_workspace_status.argtypes = [vp, vp]
     L.dmr_status_string.restype = ctypes.c_char_p
@@ -247,3 +250,16 @@ def dmr_lowbit_linear_host(X_host: torch.Tensor, q: QuantizedLinear, Y_host: tor
                                     _ptr(Y_host), out, _ptr(staging), staging.numel(), _ptr(workspace),
                                     workspace.numel(), _stream(stream)))
     return Y_host
+
+
+def dmr_lowbit_linear_noalloc(X: torch.Tensor, q: QuantizedLinear, Y: torch.Tensor, out: int = OUT_BF16, stream=None):
+    """dmr_lowbit_linear for M <= 16 without a workspace: the library's own fixed scratch is used, so
+    the call itself allocates nothing. The caller passes the output tensor Y ([M][N], bf16 or fp32)."""
+    _dev(X, torch.bfloat16, "X")
+    _dev(Y, torch.float32 if out == OUT_F32 else torch.bfloat16, "Y")
+    M, K = X.shape
+    if K != q.K or tuple(Y.shape) != (M, q.N):
+        raise DmrError(1, "shape mismatch")
+    _check(lib().dmr_lowbit_linear_noalloc(_ptr(X), M, _ptr(q.qweight), _ptr(q.scales), _ptr(q.zeros), q.N, K, q.fmt,
+                                           _ptr(Y), out, _stream(stream)))
+    return Y
