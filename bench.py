@@ -300,7 +300,7 @@ def run_ours(args):
             "gpu_launches": n_launch,
             "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": per_gpu / peaks["hbm_gbs"], "traffic": None,
-                         "kernel": "decode_lowbit_kernel", "peak_source": peaks["_source"],
+                         "kernel": "decode_stream_kernel", "peak_source": peaks["_source"],
                          "us_per_launch": seconds / n_launch * 1e6,
                          "algorithmic_bytes_per_launch": step_bytes / launches_per_step},
         })
