@@ -14,8 +14,8 @@
 //
 // Inside a CTA one producer lane keeps a ring of stages full by TMA (cp.async.bulk.tensor,
 // 128-byte swizzle): the weight box and the matching activation boxes, all completing on the
-// stage's mbarrier (a routed batch is gathered into consecutive rows beforehand).  Eight consumer warps each own 32 features and one half of the step's k range; the
-// product runs on the tensor cores with the weights as the 16-row operand of mma.m16n8k16 and up
+// stage's mbarrier (a routed batch is gathered into consecutive rows beforehand).  Eight consumer
+// warps each own 32 features and one half of the step's k range; the product runs on the tensor cores with the weights as the 16-row operand of mma.m16n8k16 and up
 // to 8 (or 2 x 8) activation rows as the 8-column operand.  4-bit codes are unpacked with one
 // LOP3 per two codes ((w >> 4p) & 0x000F000F | 0x43004300 = {128 + q_p, 128 + q_{p+4}} as two
 // bf16) and one packed subtract of (128 + zero): the tensor-core operand is the exact integer
@@ -55,16 +55,6 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         "{%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// Same product with a zero accumulator operand: c = a * b.
-__device__ __forceinline__ void mma_bf16_16816_zero(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                                    uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%10,%10,%10,%10};"
-        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 
 __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
@@ -432,9 +422,15 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                             wq[r][h][3 % WW] = v.w;
                         }
                     }
-                // When every unit ends its quantization group the group sum starts from a zero
-                // accumulator operand instead of cleared registers.
-                bool fresh = CE;
+                // when every unit ends its quantization group the group sum starts from zero here
+                if (CE) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) accg[r][nt][c] = 0.f;
+                }
                 if (BITS == 4) {
                     uint32_t zoff[R][2];
 #pragma unroll
@@ -467,12 +463,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                                     av[2 + h] = bf16x2_sub(v1, zoff[r][h]);  // codes p+1, p+5
                                 }
 #pragma unroll
-                                for (int nt = 0; nt < NT; ++nt) {
-                                    if (fresh) mma_bf16_16816_zero(accg[r][nt], av[0], av[1], av[2], av[3], b0[nt], b1[nt]);
-                                    else mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], b0[nt], b1[nt]);
-                                }
+                                for (int nt = 0; nt < NT; ++nt)
+                                    mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], b0[nt], b1[nt]);
                             }
-                            fresh = false;
                         }
                 } else if (BITS == 8) {
 #pragma unroll
@@ -492,12 +485,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                                 av[2 + h] = pack_bf16x2_rn(f[2], f[3]);
                             }
 #pragma unroll
-                            for (int nt = 0; nt < NT; ++nt) {
-                                if (fresh) mma_bf16_16816_zero(accg[r][nt], av[0], av[1], av[2], av[3], xw[nt][2 * w], xw[nt][2 * w + 1]);
-                                else mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], xw[nt][2 * w], xw[nt][2 * w + 1]);
-                            }
+                            for (int nt = 0; nt < NT; ++nt)
+                                mma_bf16_16816(accg[r][nt], av[0], av[1], av[2], av[3], xw[nt][2 * w], xw[nt][2 * w + 1]);
                         }
-                        fresh = false;
                     }
                 } else {
 #pragma unroll
