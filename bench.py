@@ -34,6 +34,9 @@ METRIC = "low-bit linear: decode weight GB/s vs HBM peak; prefill TFLOP/s vs bf1
 WORKLOAD = "decode sweep, 7B-class layer (qkv, o, gate_up, down), M in {1,8,16}, INT4 g=128"
 DECODE_MS = (1, 8, 16)
 BITS, GROUP = 4, 128
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of decode_stream_kernel, mean of the four 7B-class
+# linears at M = 1 (ncu capture summarised in profiles/decode_stream_kernel_int4_g128_7b_M1.txt)
+DECODE_TRAFFIC_BYTES_PER_LAUNCH = 26.56e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -299,7 +302,7 @@ def run_ours(args):
             "clocks": dict(clocks, window="sampled from 1.5 s before the timed region (same load) to its end"),
             "gpu_launches": n_launch,
             "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": per_gpu / peaks["hbm_gbs"], "traffic": None,
+                         "frac": per_gpu / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_BYTES_PER_LAUNCH,
                          "kernel": "decode_stream_kernel", "peak_source": peaks["_source"],
                          "us_per_launch": seconds / n_launch * 1e6,
                          "algorithmic_bytes_per_launch": step_bytes / launches_per_step},
