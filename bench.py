@@ -415,6 +415,13 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
                 del X, Y
             del q
         out["prefill"] = pre
+        # all four linears at M = 8192 as one figure for the tensor-core roofline
+        fl = sum(2.0 * 8192 * N * K for N, K in inputs.LAYER_7B.values())
+        tt = sum(pre[f"{name}_M8192"]["us"] for name in inputs.LAYER_7B) * 1e-6
+        out["roofline_prefill"] = {"bound": "tensor", "achieved": fl / tt / 1e12, "peak": peaks["bf16_tflops"],
+                                   "unit": "TFLOP/s", "frac": fl / tt / 1e12 / peaks["bf16_tflops"], "traffic": None,
+                                   "kernel": "prefill_kernel", "peak_source": peaks["_source"] + " (burst)",
+                                   "workload": "7B-class layer, four linears, M=8192, INT4 g=128, bf16 out"}
 
     if "routed" in sections:
         M = 64
