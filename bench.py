@@ -470,6 +470,33 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
             del Ws
         out["dense_decode"] = den
 
+    if "crossover" in sections:
+        # 32B-class gate and down linears, INT4 g=64 and INT8 per-channel, M = 1 .. 256, 1 % outlier channels x20:
+        # where the library's dispatch (streaming kernel up to 16 rows, tensor-core kernels above) stands.
+        # The streaming family at larger M is timed by separate runs with DMR_DECODE_MAX_M=256.
+        from paper_2602_02711_b200 import QFormat as QF
+        cx = {"dispatch": f"DMR_DECODE_MAX_M={os.environ.get('DMR_DECODE_MAX_M', '16')}"}
+        for lname, (N, K) in inputs.LAYER_32B.items():
+            for fname, f5 in (("int4_g64", QF(4, 64)), ("int8_pc", QF(8, 0))):
+                Ws = [randw(N, K, 61 + c) for c in range(2)]
+                qs = [dmr.dmr_quantize(w, f5) for w in Ws]
+                del Ws
+                for M in (1, 2, 4, 8, 16, 32, 64, 128, 256):
+                    X = torch.from_numpy(inputs.activations(M, K, seed=5, index=M, outlier_frac=0.01).view(np.int16)).view(torch.bfloat16).to(dev)
+                    Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+                    ws = dmr.new_workspace(0, M, N, K, f5, dev)
+                    state = {"i": 0}
+
+                    def call():
+                        state["i"] += 1
+                        dmr.dmr_lowbit_linear(X, qs[state["i"] % 2], OUT_BF16, Y=Y, workspace=ws)
+
+                    t = timeit(call, reps=20)
+                    b = qs[0].weight_bytes()
+                    cx[f"{lname}_{fname}_M{M}"] = {"us": t * 1e6, "gbs": b / t / 1e9, "tflops": 2.0 * M * N * K / t / 1e12}
+                del qs
+        out["crossover_32b"] = cx
+
     if "quantize" in sections:
         qz = {}
         for name, (N, K) in inputs.LAYER_7B.items():
@@ -487,7 +514,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize")
+    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

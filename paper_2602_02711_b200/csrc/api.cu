@@ -1,6 +1,7 @@
 // C ABI of libdmr: argument validation, kernel-family choice and workspace carving.
 // Every entry point validates first and launches afterwards; nothing here synchronises the host
 // except dmr_workspace_status.
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -27,7 +28,19 @@ struct Scratch {
     size_t bytes = 0;
 };
 
-bool use_gemm(int M, int N, int K, int bits, int g) { return gemm_supported(M, N, K, bits, g); }
+// Batches of up to this many rows stay on the streaming decode kernel (in chunks of 16 rows).  The
+// default is 32 (two chunks; measured faster than the tensor-core kernels up to there); the environment variable DMR_DECODE_MAX_M moves the crossover for measurements.
+int decode_max_m() {
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("DMR_DECODE_MAX_M");
+        const int x = e ? atoi(e) : 32;
+        v = x < 16 ? 16 : x;
+    }
+    return v;
+}
+
+bool use_gemm(int M, int N, int K, int bits, int g) { return M > decode_max_m() && gemm_supported(M, N, K, bits, g); }
 
 Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f) {
     Scratch s;

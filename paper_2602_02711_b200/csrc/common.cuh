@@ -70,7 +70,7 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
                            const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
                            void *scratch, int32_t *status, cudaStream_t st);
 
-// Persistent prefill GEMM (M > 128, low-bit weights): X holds M rows (for a routed call the gathered rows,
+// Persistent prefill GEMM (M > 32, low-bit weights): X holds M rows (for a routed call the gathered rows,
 // sel.count of them valid; sel.idx maps batch slots to output rows).
 bool prefill_supported(int M, int N, int K, int bits, int g);
 dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qweight, const uint16_t *scales,

@@ -331,6 +331,7 @@ int prefill_sm_count() {
 // Activation rows per tile: 256 halves the unpack work and shared-memory traffic per flop, 128 fills
 // the last wave better when there are few tiles.  Depends on (M, N) only.
 int prefill_bn(int M, int N, int sms) {
+    if (M <= 128) return 128;  // one tile of rows: the smaller activation tile leaves room for more stages
     const int n_tiles = (N + PM - 1) / PM;
     auto score = [&](int bn, double rate) {
         const long long t = (long long)n_tiles * ((M + bn - 1) / bn);
@@ -343,8 +344,11 @@ int prefill_bn(int M, int N, int sms) {
 }  // namespace
 
 bool prefill_supported(int M, int N, int K, int bits, int g) {
-    (void)N;
-    return M > 128 && (bits == 4 || bits == 8) && K % PK == 0 && g % PK == 0;
+    if (!((bits == 4 || bits == 8) && K % PK == 0 && g % PK == 0)) return false;
+    if (M > 128) return true;
+    // one tile of rows: only when the feature tiles alone fill most of the SMs (no split-K here; the
+    // split-K kernel takes the layers with few output features)
+    return M > 32 && (N + PM - 1) / PM >= 100;
 }
 
 dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qweight, const uint16_t *scales,
