@@ -220,7 +220,7 @@ def run_ours(args):
     peaks = load_peaks()
     fmt = QFormat(BITS, GROUP)
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize"}
+    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost"}
 
     def bf16_dev(bits_np):
         return torch.from_numpy(bits_np.view(np.int16)).view(torch.bfloat16).to(dev)
@@ -470,6 +470,47 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
             del Ws
         out["dense_decode"] = den
 
+    if "layer_cost" in sections:
+        # Per-token decode cost of one 7B-class layer at bf16 (T_high) and at INT4 g=128 (T_low): the four
+        # linears chained in one CUDA graph, weights rotated over copies so that they come from HBM.  The
+        # latency-based cost of the paper (Sec. 4.3, cost C = T_router N_steps + T_high N_high + T_low N_low)
+        # then gives the relative cost of a routed run at high-precision budget rho, router cost aside:
+        # C(rho) / C(all bf16) = rho + (1 - rho) T_low / T_high.
+        lc = {}
+        ncopy = 3
+        Ws = [{n: randw(N, K, 71 + 7 * c + i) for i, (n, (N, K)) in enumerate(inputs.LAYER_7B.items())} for c in range(ncopy)]
+        Qs = [{n: dmr.dmr_quantize(w, fmt) for n, w in layer.items()} for layer in Ws]
+        for M in (1, 16):
+            Xs = {n: randx(M, K, 3) for n, (N, K) in inputs.LAYER_7B.items()}
+            Ys = {n: torch.empty((M, N), dtype=torch.bfloat16, device=dev) for n, (N, K) in inputs.LAYER_7B.items()}
+            wsd = dmr.new_workspace(1, M, 22016, 11008, fmt, dev)
+            wsl = dmr.new_workspace(0, M, 22016, 11008, fmt, dev)
+            times = {}
+            for kind in ("bf16", "int4"):
+                graphs = []
+                for c in range(ncopy):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        for n in inputs.LAYER_7B:
+                            if kind == "bf16":
+                                dmr.dmr_dense_linear(Xs[n], Ws[c][n], OUT_BF16, Y=Ys[n], workspace=wsd)
+                            else:
+                                dmr.dmr_lowbit_linear(Xs[n], Qs[c][n], OUT_BF16, Y=Ys[n], workspace=wsl)
+                    graphs.append(g)
+                state = {"i": 0}
+
+                def call():
+                    state["i"] += 1
+                    graphs[state["i"] % ncopy].replay()
+
+                times[kind] = timeit(call, reps=60)
+            ratio = times["int4"] / times["bf16"]
+            lc[f"M{M}"] = {"t_high_us_per_layer": times["bf16"] * 1e6, "t_low_us_per_layer": times["int4"] * 1e6,
+                           "t_high_over_t_low": 1.0 / ratio,
+                           "relative_cost_at_budget": {f"rho={r}": r + (1 - r) * ratio for r in (0.2, 0.4, 0.7)}}
+        del Ws, Qs
+        out["layer_cost_7b"] = lc
+
     if "crossover" in sections:
         # 32B-class gate and down linears, INT4 g=64 and INT8 per-channel, M = 1 .. 256, 1 % outlier channels x20:
         # where the library's dispatch (streaming kernel up to 16 rows, tensor-core kernels above) stands.
@@ -514,7 +555,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover")
+    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
