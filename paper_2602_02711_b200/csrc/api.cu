@@ -22,6 +22,7 @@ struct Scratch {
     int32_t *status = nullptr;
     int32_t *counts = nullptr, *idx_high = nullptr, *idx_low = nullptr;
     uint16_t *xg_low = nullptr, *xg_high = nullptr;
+    void *prefill_scratch = nullptr;  // prepared fp16 activations and row scales of the prefill kernel
     float *partial = nullptr;
     void *stream_scratch = nullptr;  // counters + partial sums of the streaming decode kernel
     uint16_t *xg_stream = nullptr;   // routed, decode path: 16 gathered activation rows
@@ -66,6 +67,10 @@ Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f
             off += xg;
         }
     }
+    if (low_gemm && prefill_supported(M, N, K, f.bits, g)) {
+        s.prefill_scratch = base + off;
+        off += round_up(prefill_scratch_bytes(M, K), 256);
+    }
     size_t partial = 0;
     if (low_gemm) partial = gemm_plan(M, N, K, f.bits).partial_bytes;
     if (dense_gemm) {
@@ -107,14 +112,14 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
     const int g = group_of(K, f);
     const size_t ysz = out == DMR_OUT_F32 ? 4 : 2;
     if (use_gemm(M, N, K, f.bits, g)) {
+        if (prefill_supported(M, N, K, f.bits, g))  // gathers the listed rows itself
+            return launch_prefill(X, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.prefill_scratch, ws.status, st);
         const uint16_t *Xin = X;
         if (sel.idx) {
             dmr_status_t r = launch_gather_rows(X, K, M, sel.idx, sel.count, 0, ws.xg_low, st);
             if (r != DMR_OK) return r;
             Xin = ws.xg_low;
         }
-        if (prefill_supported(M, N, K, f.bits, g))
-            return launch_prefill(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.status, st);
         return launch_gemm(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.partial, ws.status, st);
     }
     if (!stream_supported(M < 16 ? M : 16, N, K, f.bits, g))

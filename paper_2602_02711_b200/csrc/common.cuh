@@ -70,12 +70,15 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
                            const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
                            void *scratch, int32_t *status, cudaStream_t st);
 
-// Persistent prefill GEMM (M > 32, low-bit weights): X holds M rows (for a routed call the gathered rows,
-// sel.count of them valid; sel.idx maps batch slots to output rows).
+// Persistent prefill GEMM (M > 32, low-bit weights); sel.idx maps batch slots to rows of X and Y, sel.count
+// says how many slots are valid.
 bool prefill_supported(int M, int N, int K, int bits, int g);
+// X is the caller's activation matrix (for a routed call the rows sel.idx lists are gathered);
+// `scratch` holds prefill_scratch_bytes(M, K) bytes for the prepared fp16 activations and their row scales.
+size_t prefill_scratch_bytes(int M, int K);
 dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qweight, const uint16_t *scales,
                             const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
-                            int32_t *status, cudaStream_t st);
+                            void *scratch, int32_t *status, cudaStream_t st);
 
 // Tensor-core GEMM family (M > 16): tcgen05 MMA with TMA-staged operands.
 struct GemmPlan {

@@ -9,14 +9,22 @@
 // Per 64-wide k block and stage of the ring:
 //   warp 0      TMA: the packed code tile [128 features x 32 or 64 bytes] and the activation tile
 //               [BN rows x 128 bytes, 128-byte swizzle] land in shared memory (one mbarrier);
-//   warps 2..5  one thread per feature row turns its codes into the bf16 weights s * (q - zero)
-//               (exact integer q - zero, then ONE rounding of the product: the nearest bf16 of
-//               the dequantized weight) and stores them as the swizzled K-major A tile;
+//   warps 2..5  one thread per feature row turns its codes into the fp16 weights s' * (q - zero)
+//               (exact integer q - zero, then ONE rounding of the product to 11 significant bits)
+//               and stores them as the swizzled K-major A tile;
 //   warp 1      one lane issues four tcgen05.mma (128 x BN x 16) that accumulate into one of two
 //               fp32 accumulators in tensor memory, and commits the stage back to the producer;
 //   warps 6..9  drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
 //               next tile's MMAs run into the other accumulator.
 // CTAs are persistent: CTA b takes tiles b, b + grid, ...  Every wait is bounded.
+//
+// Operand precision.  The MMA runs in fp16 x fp16 -> fp32 (kind::f16) instead of bf16: a bf16 A
+// operand would round every dequantized weight to 8 significant bits (1.5e-3 rms relative error of
+// the outputs, uncomfortably close to the 2e-3 acceptance bound), fp16 keeps 11 (1.8e-4).  To stay
+// inside fp16's range whatever the inputs, a preparation kernel rescales every activation row by a
+// power of two (row maximum into [2^13, 2^14): exact for all elements within 2^-27 of the maximum)
+// and the unpack threads rescale a feature's scales by the power of two of its largest one; the
+// epilogue multiplies the two powers of two back in (exact).
 #include <cuda_bf16.h>
 
 #include "sm100.cuh"
@@ -30,7 +38,7 @@ constexpr int PK = 64;   // k per stage
 
 template <int BITS, int BN>
 struct PrefillCfg {
-    static constexpr int A_BYTES = PM * PK * 2;              // 16 KB of bf16 weights
+    static constexpr int A_BYTES = PM * PK * 2;              // 16 KB of fp16 weights
     static constexpr int B_BYTES = BN * PK * 2;              // activations
     static constexpr int P_ROW = PK * BITS / 8;              // packed bytes per feature per stage
     static constexpr int P_BYTES = PM * P_ROW;               // 4 or 8 KB
@@ -45,6 +53,7 @@ struct PrefillCfg {
 struct PrefillArgs {
     const uint16_t *scales;
     const uint8_t *zeros;
+    const float *xscale;   // power of two each prepared activation row was divided by
     void *Y;
     const int32_t *idx;    // routed: output row of batch slot m (nullptr = identity)
     const int32_t *count;  // routed: number of valid slots (nullptr = M)
@@ -63,20 +72,99 @@ __device__ __forceinline__ uint32_t p_prmt(uint32_t a, uint32_t b, uint32_t sel)
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
     return r;
 }
-__device__ __forceinline__ uint32_t p_sub_bf16x2(uint32_t a, uint32_t b) {
+__device__ __forceinline__ uint32_t p_sub_f16x2(uint32_t a, uint32_t b) {
     uint32_t r;
-    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
     return r;
 }
-__device__ __forceinline__ uint32_t p_mul_bf16x2(uint32_t a, uint32_t b) {
+__device__ __forceinline__ uint32_t p_mul_f16x2(uint32_t a, uint32_t b) {
     uint32_t r;
-    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
     return r;
 }
-__device__ __forceinline__ uint32_t p_pack_bf16x2(float lo, float hi) {
+__device__ __forceinline__ uint32_t p_pack_f16x2(float lo, float hi) {
     uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+
+// Activation preparation: Xh[slot][k] = fp16(X[row(slot)][k] * 2^-e), xscale[slot] = 2^e, with e chosen
+// per row so that the row's largest magnitude lands in [2^13, 2^14).  One warp per slot; slots past
+// the valid count (routed calls) are zero-filled.  `idx` / `count` as in the GEMM (nullptr = identity).
+// REG: the row (K <= 4096) is held in registers between the two passes, so it is read once.
+__device__ __forceinline__ uint32_t row_max_bits(const uint4 &q, uint32_t mx) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t a0 = w[i] & 0x7FFFu, a1 = (w[i] >> 16) & 0x7FFFu;
+        if (a0 < 0x7F80u) mx = max(mx, a0);  // largest FINITE magnitude (bf16 patterns order like magnitudes)
+        if (a1 < 0x7F80u) mx = max(mx, a1);
+    }
+    return mx;
+}
+
+__device__ __forceinline__ uint4 to_f16_scaled(const uint4 &q, float down, float down2) {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float f0 = __uint_as_float(w[i] << 16) * down * down2;
+        const float f1 = __uint_as_float(w[i] & 0xFFFF0000u) * down * down2;
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(o[i]) : "f"(f1), "f"(f0));
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+template <bool REG>
+__global__ void __launch_bounds__(256)
+xprep_kernel(const uint16_t *__restrict__ X, int K, int Mcap, const int32_t *__restrict__ idx,
+             const int32_t *__restrict__ count, uint16_t *__restrict__ Xh, float *__restrict__ xscale) {
+    constexpr int CH = 16;  // 16-byte chunks per lane in the register path: K <= 32 * 16 * 8 = 4096
+    const int rows = count ? min(*count, Mcap) : Mcap;
+    const int lane = threadIdx.x & 31;
+    const int nv = K / 8;
+    for (int slot = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); slot < Mcap; slot += (int)((gridDim.x * blockDim.x) >> 5)) {
+        uint4 *dst = reinterpret_cast<uint4 *>(Xh + (size_t)slot * K);
+        if (slot >= rows) {
+            for (int v = lane; v < nv; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+            if (lane == 0) xscale[slot] = 1.f;
+            continue;
+        }
+        const uint4 *src = reinterpret_cast<const uint4 *>(X + (size_t)(idx ? idx[slot] : slot) * K);
+        uint4 keep[REG ? CH : 1];
+        uint32_t mx = 0;
+        if (REG) {
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int v = c * 32 + lane;
+                keep[c] = v < nv ? __ldg(src + v) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int c = 0; c < CH; ++c) mx = row_max_bits(keep[c], mx);
+        } else {
+#pragma unroll 4
+            for (int v = lane; v < nv; v += 32) mx = row_max_bits(__ldg(src + v), mx);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        int eb = (int)(mx >> 7);          // biased exponent of the maximum (0 for zero / subnormal rows)
+        if (eb < 1) eb = 1;
+        const int e = (eb - 127) - 13;    // x * 2^-e has its maximum in [2^13, 2^14)
+        // 2^-e as one or two float factors (|e| can reach 139, beyond one float exponent)
+        const float down = e > 0 ? __uint_as_float((uint32_t)(127 - min(e, 126)) << 23) : __uint_as_float((uint32_t)(127 + min(-e, 127)) << 23);
+        const float down2 = e < -127 ? __uint_as_float((uint32_t)(127 + (-e - 127)) << 23) : 1.f;
+        if (REG) {
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int v = c * 32 + lane;
+                if (v < nv) dst[v] = to_f16_scaled(keep[c], down, down2);
+            }
+        } else {
+#pragma unroll 4
+            for (int v = lane; v < nv; v += 32) dst[v] = to_f16_scaled(__ldg(src + v), down, down2);
+        }
+        if (lane == 0) xscale[slot] = ldexpf(1.f, e);
+    }
 }
 
 template <int BITS, int BN, bool OUT_F32>
@@ -154,7 +242,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            constexpr uint32_t IDESC = umma_idesc_bf16(PM, BN);
+            constexpr uint32_t IDESC = umma_idesc_f16(PM, BN);
             uint32_t it = 0, tile_it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
@@ -180,7 +268,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
         }
     } else if (warp < 6) {
-        // ================= unpack warps: codes -> bf16 weights s * (q - zero) =================
+        // ================= unpack warps: codes -> fp16 weights s' * (q - zero) =================
         const int r = (warp - 2) * 32 + lane;  // feature row of the tile
         const uint32_t swz = (uint32_t)(r & 7);
         uint32_t it = 0;
@@ -189,6 +277,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const int n = min((tile % a.n_tiles) * PM + r, a.N - 1);
             const uint16_t *sp = a.scales + (size_t)n * G;
             const uint8_t *zp = a.zeros + (size_t)n * G;
+            // power of two of the feature's largest scale: s' = s * 2^-f lies in (0, 2)
+            uint32_t smax = 0;
+            for (int gi = 0; gi < G; ++gi) smax = max(smax, (uint32_t)__ldg(sp + gi) & 0x7FFFu);
+            int fb = (int)(smax >> 7);
+            fb = fb < 1 ? 1 : (fb > 253 ? 253 : fb);
+            const float fdown = __uint_as_float((uint32_t)(254 - fb) << 23);  // 2^-(fb - 127)
             uint32_t sb = __ldg(sp), zb = __ldg(zp);
             for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % S;
@@ -209,15 +303,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     uint32_t w[8];
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(src));
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(src + 16));
-                    const uint32_t zz = 0x4300u | zb;             // bf16 of 128 + zero
-                    const uint32_t zoff = zz | (zz << 16);
-                    const uint32_t s2 = sb | (sb << 16);          // the bf16 scale twice
+                    // fp16 patterns: 0x6400 | q = 1024 + q and 0x6400 | (q << 4) = 1024 + 16 q (no shift needed
+                    // for the odd codes); minus 1024 + zero (or 1024 + 16 zero) is exact; then one rounding
+                    const float sf = __uint_as_float(sb << 16) * fdown;
+                    uint32_t s2, s2_16;
+                    asm("cvt.rn.f16x2.f32 %0, %1, %1;" : "=r"(s2) : "f"(sf));
+                    asm("cvt.rn.f16x2.f32 %0, %1, %1;" : "=r"(s2_16) : "f"(sf * 0.0625f));
+                    const uint32_t zz = 0x6400u | zb, zz16 = 0x6400u | (zb << 4);
+                    const uint32_t zoff = zz | (zz << 16), zoff16 = zz16 | (zz16 << 16);
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {  // word c = codes 8c .. 8c+7 = 16-byte chunk c of the row
-                        const uint32_t d04 = p_mul_bf16x2(p_sub_bf16x2(p_lop3_and_or(w[c], 0x000F000Fu, 0x43004300u), zoff), s2);
-                        const uint32_t d15 = p_mul_bf16x2(p_sub_bf16x2(p_lop3_and_or(w[c] >> 4, 0x000F000Fu, 0x43004300u), zoff), s2);
-                        const uint32_t d26 = p_mul_bf16x2(p_sub_bf16x2(p_lop3_and_or(w[c] >> 8, 0x000F000Fu, 0x43004300u), zoff), s2);
-                        const uint32_t d37 = p_mul_bf16x2(p_sub_bf16x2(p_lop3_and_or(w[c] >> 12, 0x000F000Fu, 0x43004300u), zoff), s2);
+                        const uint32_t w8 = w[c] >> 8;
+                        const uint32_t d04 = p_mul_f16x2(p_sub_f16x2(p_lop3_and_or(w[c], 0x000F000Fu, 0x64006400u), zoff), s2);
+                        const uint32_t d15 = p_mul_f16x2(p_sub_f16x2(p_lop3_and_or(w[c], 0x00F000F0u, 0x64006400u), zoff16), s2_16);
+                        const uint32_t d26 = p_mul_f16x2(p_sub_f16x2(p_lop3_and_or(w8, 0x000F000Fu, 0x64006400u), zoff), s2);
+                        const uint32_t d37 = p_mul_f16x2(p_sub_f16x2(p_lop3_and_or(w8, 0x00F000F0u, 0x64006400u), zoff16), s2_16);
                         const uint32_t o01 = p_prmt(d04, d15, 0x5410), o45 = p_prmt(d04, d15, 0x7632);
                         const uint32_t o23 = p_prmt(d26, d37, 0x5410), o67 = p_prmt(d26, d37, 0x7632);
                         const uint32_t addr = dst + ((((uint32_t)c) ^ swz) << 4);
@@ -225,7 +325,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                 } else {
                     const float zf = __uint_as_float(0x4B000000u | zb);  // 2^23 + zero
-                    const float sf = __uint_as_float(sb << 16);
+                    const float sf = __uint_as_float(sb << 16) * fdown;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {  // chunk c = codes 8c .. 8c+7 = packed words 2c, 2c+1
                         uint32_t w0, w1;
@@ -238,8 +338,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                             for (int b = 0; b < 4; ++b)  // (q - zero) exactly, times the scale exactly (8 x 8 bits)
                                 f[b] = __fmul_rn(__fsub_rn(__uint_as_float(p_prmt(u, 0x4B000000u, 0x7650u + (uint32_t)b)), zf), sf);
-                            o[2 * h] = p_pack_bf16x2(f[0], f[1]);  // the one rounding
-                            o[2 * h + 1] = p_pack_bf16x2(f[2], f[3]);
+                            o[2 * h] = p_pack_f16x2(f[0], f[1]);  // the one rounding
+                            o[2 * h + 1] = p_pack_f16x2(f[2], f[3]);
                         }
                         const uint32_t addr = dst + ((((uint32_t)c) ^ swz) << 4);
                         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
@@ -261,6 +361,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
             const int buf = tile_it & 1;
             const int n = (tile % a.n_tiles) * PM + r, m0 = (tile / a.n_tiles) * BN;
+            // the power of two the unpack threads divided this feature's scales by, undone here
+            uint32_t smax = 0;
+            {
+                const uint16_t *sp = a.scales + (size_t)min(n, a.N - 1) * G;
+                for (int gi = 0; gi < G; ++gi) smax = max(smax, (uint32_t)__ldg(sp + gi) & 0x7FFFu);
+            }
+            int fb = (int)(smax >> 7);
+            fb = fb < 1 ? 1 : (fb > 253 ? 253 : fb);
+            const float fscale = __uint_as_float((uint32_t)fb << 23);  // 2^(fb - 127)
             if (!mbar_wait(tfull_bar(buf), (tile_it >> 1) & 1, a.status)) break;
             tcgen05_fence_after();
 #pragma unroll 1
@@ -280,7 +389,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         const int m = m0 + c0 + c;
                         if (m < rows) {
                             const int row = a.idx ? a.idx[m] : m;
-                            const float v = __uint_as_float(u[c]);
+                            const float v = (__uint_as_float(u[c]) * __ldg(a.xscale + m)) * fscale;
                             if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
                             else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
                         }
@@ -351,13 +460,26 @@ bool prefill_supported(int M, int N, int K, int bits, int g) {
     return M > 32 && (N + PM - 1) / PM >= 100;
 }
 
+size_t prefill_scratch_bytes(int M, int K) { return round_up((size_t)M * K * 2, 256) + round_up((size_t)M * 4, 256); }
+
 dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qweight, const uint16_t *scales,
                             const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
-                            int32_t *status, cudaStream_t st) {
+                            void *scratch, int32_t *status, cudaStream_t st) {
     const int sms = prefill_sm_count();
     const int bn = prefill_bn(M, N, sms);
+    // activations: gather (routed calls), rescale each row by a power of two and convert to fp16
+    uint16_t *Xh = reinterpret_cast<uint16_t *>(scratch);
+    float *xscale = reinterpret_cast<float *>(reinterpret_cast<char *>(scratch) + round_up((size_t)M * K * 2, 256));
+    {
+        int blocks = (M + 7) / 8;
+        if (blocks > sms * 8) blocks = sms * 8;
+        if (K <= 4096) xprep_kernel<true><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
+        else xprep_kernel<false><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
+        dmr_status_t r = check_launch();
+        if (r != DMR_OK) return r;
+    }
     CUtensorMap map_w, map_x;
-    if (!make_tensor_map_2d(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)K * 2,
+    if (!make_tensor_map_2d(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Xh, (uint64_t)M, (uint64_t)K, (uint64_t)K * 2,
                             (uint32_t)bn, PK, TmaSwizzle::k128B))
         return DMR_ERR_CUDA;
     const uint64_t row_bytes = (uint64_t)K * bits / 8;
@@ -367,6 +489,7 @@ dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qw
     PrefillArgs a;
     a.scales = scales;
     a.zeros = zeros;
+    a.xscale = xscale;
     a.Y = Y;
     a.idx = sel.idx;
     a.count = sel.count;

@@ -178,6 +178,11 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t addr) {
 }
 
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+// The same with both operands fp16.
+__host__ __device__ constexpr uint32_t umma_idesc_f16(int m, int n) {
+    return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
