@@ -89,9 +89,8 @@ __device__ __forceinline__ uint32_t p_pack_f16x2(float lo, float hi) {
 }
 
 // Activation preparation: Xh[slot][k] = fp16(X[row(slot)][k] * 2^-e), xscale[slot] = 2^e, with e chosen
-// per row so that the row's largest magnitude lands in [2^13, 2^14).  One warp per slot; slots past
-// the valid count (routed calls) are zero-filled.  `idx` / `count` as in the GEMM (nullptr = identity).
-// REG: the row (K <= 4096) is held in registers between the two passes, so it is read once.
+// per row so that the row's largest magnitude lands in [2^13, 2^14).  Slots past the valid count
+// (routed calls) are zero-filled.  `idx` / `count` as in the GEMM (nullptr = identity).
 __device__ __forceinline__ uint32_t row_max_bits(const uint4 &q, uint32_t mx) {
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
@@ -115,55 +114,52 @@ __device__ __forceinline__ uint4 to_f16_scaled(const uint4 &q, float down, float
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-template <bool REG>
+// One CTA of 256 threads per slot (grid-stride over slots); CH = 16-byte chunks a thread keeps in
+// registers between the two passes (CH * 256 * 8 >= K), so the row is read from memory once.
+template <int CH>
 __global__ void __launch_bounds__(256)
 xprep_kernel(const uint16_t *__restrict__ X, int K, int Mcap, const int32_t *__restrict__ idx,
              const int32_t *__restrict__ count, uint16_t *__restrict__ Xh, float *__restrict__ xscale) {
-    constexpr int CH = 16;  // 16-byte chunks per lane in the register path: K <= 32 * 16 * 8 = 4096
+    __shared__ uint32_t warp_max[8];
     const int rows = count ? min(*count, Mcap) : Mcap;
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nv = K / 8;
-    for (int slot = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); slot < Mcap; slot += (int)((gridDim.x * blockDim.x) >> 5)) {
+    for (int slot = blockIdx.x; slot < Mcap; slot += gridDim.x) {
         uint4 *dst = reinterpret_cast<uint4 *>(Xh + (size_t)slot * K);
         if (slot >= rows) {
-            for (int v = lane; v < nv; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
-            if (lane == 0) xscale[slot] = 1.f;
+            for (int v = threadIdx.x; v < nv; v += 256) dst[v] = make_uint4(0, 0, 0, 0);
+            if (threadIdx.x == 0) xscale[slot] = 1.f;
             continue;
         }
         const uint4 *src = reinterpret_cast<const uint4 *>(X + (size_t)(idx ? idx[slot] : slot) * K);
-        uint4 keep[REG ? CH : 1];
+        uint4 keep[CH];
         uint32_t mx = 0;
-        if (REG) {
 #pragma unroll
-            for (int c = 0; c < CH; ++c) {
-                const int v = c * 32 + lane;
-                keep[c] = v < nv ? __ldg(src + v) : make_uint4(0, 0, 0, 0);
-            }
-#pragma unroll
-            for (int c = 0; c < CH; ++c) mx = row_max_bits(keep[c], mx);
-        } else {
-#pragma unroll 4
-            for (int v = lane; v < nv; v += 32) mx = row_max_bits(__ldg(src + v), mx);
+        for (int c = 0; c < CH; ++c) {
+            const int v = c * 256 + threadIdx.x;
+            keep[c] = v < nv ? __ldg(src + v) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
+        for (int c = 0; c < CH; ++c) mx = row_max_bits(keep[c], mx);
+#pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        __syncthreads();  // warp_max of the previous slot has been read by everyone
+        if (lane == 0) warp_max[warp] = mx;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < 8; ++w) mx = max(mx, warp_max[w]);
         int eb = (int)(mx >> 7);          // biased exponent of the maximum (0 for zero / subnormal rows)
         if (eb < 1) eb = 1;
         const int e = (eb - 127) - 13;    // x * 2^-e has its maximum in [2^13, 2^14)
         // 2^-e as one or two float factors (|e| can reach 139, beyond one float exponent)
         const float down = e > 0 ? __uint_as_float((uint32_t)(127 - min(e, 126)) << 23) : __uint_as_float((uint32_t)(127 + min(-e, 127)) << 23);
         const float down2 = e < -127 ? __uint_as_float((uint32_t)(127 + (-e - 127)) << 23) : 1.f;
-        if (REG) {
 #pragma unroll
-            for (int c = 0; c < CH; ++c) {
-                const int v = c * 32 + lane;
-                if (v < nv) dst[v] = to_f16_scaled(keep[c], down, down2);
-            }
-        } else {
-#pragma unroll 4
-            for (int v = lane; v < nv; v += 32) dst[v] = to_f16_scaled(__ldg(src + v), down, down2);
+        for (int c = 0; c < CH; ++c) {
+            const int v = c * 256 + threadIdx.x;
+            if (v < nv) dst[v] = to_f16_scaled(keep[c], down, down2);
         }
-        if (lane == 0) xscale[slot] = ldexpf(1.f, e);
+        if (threadIdx.x == 0) xscale[slot] = ldexpf(1.f, e);
     }
 }
 
@@ -453,7 +449,7 @@ int prefill_bn(int M, int N, int sms) {
 }  // namespace
 
 bool prefill_supported(int M, int N, int K, int bits, int g) {
-    if (!((bits == 4 || bits == 8) && K % PK == 0 && g % PK == 0)) return false;
+    if (!((bits == 4 || bits == 8) && K % PK == 0 && g % PK == 0 && K <= 32768)) return false;
     if (M > 128) return true;
     // one tile of rows: only when the feature tiles alone fill most of the SMs (no split-K here; the
     // split-K kernel takes the layers with few output features)
@@ -471,10 +467,11 @@ dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qw
     uint16_t *Xh = reinterpret_cast<uint16_t *>(scratch);
     float *xscale = reinterpret_cast<float *>(reinterpret_cast<char *>(scratch) + round_up((size_t)M * K * 2, 256));
     {
-        int blocks = (M + 7) / 8;
-        if (blocks > sms * 8) blocks = sms * 8;
-        if (K <= 4096) xprep_kernel<true><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
-        else xprep_kernel<false><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
+        const int blocks = M < sms * 16 ? M : sms * 16;
+        if (K <= 2 * 2048) xprep_kernel<2><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
+        else if (K <= 8 * 2048) xprep_kernel<8><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
+        else if (K <= 16 * 2048) xprep_kernel<16><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
+        else return DMR_ERR_UNSUPPORTED;
         dmr_status_t r = check_launch();
         if (r != DMR_OK) return r;
     }
