@@ -114,7 +114,10 @@ dmr_status_t dmr_dense_linear(const void *X_bf16, int M, const void *W_bf16, int
  * with the bf16 weights W, the others with the low-bit weights; every row's result is written
  * at its own index m, so Y is in step order.  The mask is read on the device only.  Row m equals,
  * bit for bit, row m of dmr_dense_linear (mask != 0) or dmr_lowbit_linear (mask == 0) called
- * on the same M rows.
+ * on the same M rows.  The two halves run concurrently: the library forks a helper stream after the
+ * partition and joins it back into `stream` before returning (also under stream capture).  The
+ * helper stream and its two events are created by the first routed call on a device; make that
+ * first call outside any capture.
  */
 dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, const void *W_bf16,
                                const void *qweight, const void *scales, const void *zeros, int N,

@@ -26,6 +26,10 @@ struct Scratch {
     float *partial = nullptr;
     void *stream_scratch = nullptr;  // counters + partial sums of the streaming decode kernel
     uint16_t *xg_stream = nullptr;   // routed, decode path: 16 gathered activation rows
+    // routed calls run their two halves on two streams: the high-precision half gets its own scratch
+    float *partial_high = nullptr;
+    void *stream_scratch_high = nullptr;
+    uint16_t *xg_stream_high = nullptr;
     size_t bytes = 0;
 };
 
@@ -71,15 +75,20 @@ Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f
         s.prefill_scratch = base + off;
         off += round_up(prefill_scratch_bytes(M, K), 256);
     }
-    size_t partial = 0;
-    if (low_gemm) partial = gemm_plan(M, N, K, f.bits).partial_bytes;
-    if (dense_gemm) {
-        const size_t p2 = gemm_plan(M, N, K, 0).partial_bytes;
-        if (p2 > partial) partial = p2;
-    }
-    if (partial) {
+    const size_t partial_low = low_gemm ? gemm_plan(M, N, K, f.bits).partial_bytes : 0;
+    const size_t partial_dense = dense_gemm ? gemm_plan(M, N, K, 0).partial_bytes : 0;
+    if (op == DMR_OP_ROUTED_LINEAR) {
+        if (partial_low) {
+            s.partial = reinterpret_cast<float *>(base + off);
+            off += round_up(partial_low, 256);
+        }
+        if (partial_dense) {
+            s.partial_high = reinterpret_cast<float *>(base + off);
+            off += round_up(partial_dense, 256);
+        }
+    } else if (partial_low || partial_dense) {
         s.partial = reinterpret_cast<float *>(base + off);
-        off += round_up(partial, 256);
+        off += round_up(partial_low > partial_dense ? partial_low : partial_dense, 256);
     }
     const bool low_stream = op != DMR_OP_DENSE_LINEAR && !low_gemm;
     const bool dense_stream = op != DMR_OP_LOWBIT_LINEAR && !dense_gemm;
@@ -88,6 +97,10 @@ Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f
         off += round_up(stream_scratch_bytes(N), 256);
         if (op == DMR_OP_ROUTED_LINEAR) {
             s.xg_stream = reinterpret_cast<uint16_t *>(base + off);
+            off += round_up((size_t)16 * K * 2, 256);
+            s.stream_scratch_high = base + off;
+            off += round_up(stream_scratch_bytes(N), 256);
+            s.xg_stream_high = reinterpret_cast<uint16_t *>(base + off);
             off += round_up((size_t)16 * K * 2, 256);
         }
     }
@@ -182,6 +195,31 @@ dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, 
         if (r != DMR_OK) return r;
     }
     return DMR_OK;
+}
+
+// Helper stream and fork / join events of the routed call, one set per device, created at the first
+// routed call on that device (so make that first call outside any stream capture).
+struct SideStream {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+
+SideStream *side_stream() {
+    static SideStream per_device[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    SideStream &s = per_device[dev];
+    if (!s.stream) {
+        cudaError_t e = cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            s.stream = nullptr;
+            return nullptr;
+        }
+    }
+    return &s;
 }
 
 }  // namespace
@@ -295,12 +333,35 @@ dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, c
     r = launch_route_partition(mask, M, ws.idx_high, ws.idx_low, ws.counts, st);
     if (r != DMR_OK) return r;
     const uint16_t *X = reinterpret_cast<const uint16_t *>(X_bf16);
-    RowSel low = {ws.idx_low, ws.counts + 1, 0};
-    r = run_lowbit(X, M, low, reinterpret_cast<const uint32_t *>(qweight), reinterpret_cast<const uint16_t *>(scales),
-                   reinterpret_cast<const uint8_t *>(zeros), N, K, f, Y, out, ws, st);
-    if (r != DMR_OK) return r;
+    // the two halves touch different rows of Y and different scratch: the high-precision half runs on a
+    // helper stream, forked after the partition and joined before the call's work on `stream` ends
+    SideStream *side = side_stream();
+    if (!side) return DMR_ERR_CUDA;
+    cudaError_t e = cudaEventRecord(side->fork, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(side->stream, side->fork, 0);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return DMR_ERR_CUDA;
+    }
+    Scratch wh = ws;
+    wh.partial = ws.partial_high;
+    wh.stream_scratch = ws.stream_scratch_high;
+    wh.xg_stream = ws.xg_stream_high;
     RowSel high = {ws.idx_high, ws.counts + 0, 0};
-    return run_dense(X, M, high, reinterpret_cast<const uint16_t *>(W_bf16), N, K, Y, out, ws, st);
+    const dmr_status_t rh = run_dense(X, M, high, reinterpret_cast<const uint16_t *>(W_bf16), N, K, Y, out, wh, side->stream);
+    RowSel low = {ws.idx_low, ws.counts + 1, 0};
+    const dmr_status_t rl = run_lowbit(X, M, low, reinterpret_cast<const uint32_t *>(qweight), reinterpret_cast<const uint16_t *>(scales),
+                                       reinterpret_cast<const uint8_t *>(zeros), N, K, f, Y, out, ws, st);
+    // always join, also after an error, so that the helper stream never outlives the call (or a capture)
+    e = cudaEventRecord(side->join, side->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join, 0);
+    if (rh != DMR_OK) return rh;
+    if (rl != DMR_OK) return rl;
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return DMR_ERR_CUDA;
+    }
+    return DMR_OK;
 }
 
 size_t dmr_host_staging_bytes(int M, int N, int K, dmr_out_t out) {
