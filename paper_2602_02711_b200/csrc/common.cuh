@@ -64,6 +64,9 @@ dmr_status_t launch_dequantize(const uint32_t *qweight, const uint16_t *scales, 
 // for packed codes and 16 for bf16 weights.  `scratch` holds stream_scratch_bytes(N) bytes that are
 // zero before the first use (the kernel leaves its counters zeroed again).
 constexpr int kMaxStreamCtas = 512;
+// Feature-group counters sit one per 128-byte line: counts into different groups then never queue up
+// behind each other in the L2.
+constexpr int kCounterStride = 32;  // int32 words between counters
 size_t stream_scratch_bytes(int N);
 bool stream_supported(int M, int N, int K, int bits, int g);
 dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,

@@ -17,7 +17,7 @@ namespace {
 constexpr int kNoallocMaxN = 65536;
 constexpr size_t kNoallocStatusBytes = 256;
 constexpr size_t kNoallocScratchBytes =
-    kNoallocStatusBytes + ((size_t)(kNoallocMaxN / 128) * sizeof(int32_t) + 255) / 256 * 256 +
+    kNoallocStatusBytes + (size_t)(kNoallocMaxN / 128) * kCounterStride * sizeof(int32_t) +
     (size_t)kMaxStreamCtas * 2 * 16 * 128 * sizeof(float);
 
 // In host code this name is only a handle for cudaGetSymbolAddress, never a device address.

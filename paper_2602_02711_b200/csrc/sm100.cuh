@@ -80,7 +80,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
 // The same bounded wait for a thread that has nothing to do until the phase completes and shares
 // its scheduler with busy warps: the hardware may suspend it for up to `suspend_ns` per try, and
 // it sleeps between tries instead of spinning, so that it takes almost no issue slots.
-__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, int32_t *status, uint32_t suspend_ns = 2000) {
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, int32_t *status, uint32_t suspend_ns = 2000,
+                                               uint32_t sleep_ns = 100) {
     for (uint32_t i = 0; i < (kWaitLimit >> 4); ++i) {
         uint32_t ok;
         asm volatile(
@@ -91,7 +92,7 @@ __device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, in
             : "r"(bar), "r"(parity), "r"(suspend_ns)
             : "memory");
         if (ok) return true;
-        __nanosleep(100);
+        __nanosleep(sleep_ns);
     }
     if (status) atomicExch(status, (int32_t)DMR_ERR_TIMEOUT);
     return false;

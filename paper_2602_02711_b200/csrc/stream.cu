@@ -10,7 +10,10 @@
 // the shape.  A feature group whose steps are shared by several CTAs is finished by the last of
 // them to arrive, which adds the partial sums in CTA order (no floating-point atomics), so the
 // summation order of an output depends on (N, K) and the SM count only - never on M, on the
-// row's position in the batch or on the other rows.
+// row's position in the batch or on the other rows.  Counting a CTA into a shared group costs two
+// round trips to the L2 (fence, atomic); one lane of a warp of its own does that while the consumer
+// warps go on with their next steps, and the sums of the groups a CTA was last for are formed at
+// the end of the kernel by all consumer warps.
 //
 // Inside a CTA one producer lane keeps a ring of stages full by TMA (cp.async.bulk.tensor,
 // 128-byte swizzle): the weight box and the matching activation boxes, all completing on the
@@ -39,14 +42,13 @@ namespace {
 constexpr int kR = 2;                                        // 16-feature tiles per consumer warp
 constexpr int kRowBlocks = 128 / (16 * kR);                  // consumer warps side by side over the features
 constexpr int kConsumerWarps = 2 * kRowBlocks;               // two k halves
-constexpr int kStreamThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
+constexpr int kPublishWarp = kConsumerWarps + 1;            // one lane counts this CTA into shared feature groups
+constexpr int kStreamThreads = (kConsumerWarps + 2) * 32;  // + one producer warp + the publishing warp
 constexpr int kTileRows = 128;                              // features per step
 constexpr int kStepBytes = kTileRows * 128;                 // weight bytes per step (16 KB)
 constexpr int kMaxStages = 12;
-#ifndef DMR_STAGE_BUDGET_KB
-#define DMR_STAGE_BUDGET_KB 100
-#endif
-constexpr int kStageBudget = DMR_STAGE_BUDGET_KB;          // shared memory for the stage ring, KB
+// Shared memory for the stage ring, KB: two 8-row CTAs share an SM, a 16-row CTA has it alone.
+__host__ __device__ constexpr int stage_budget_kb(int nt) { return nt == 1 ? 92 : 100; }
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                                uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -93,6 +95,7 @@ __device__ __forceinline__ uint2 lds64(uint32_t addr) {
     return v;
 }
 
+__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -109,17 +112,19 @@ struct StepGeom {
     static constexpr int X_BOXES = STEP_K / 64;        // activation boxes of 64 k (128 bytes per row): 4, 2, 1
 };
 
-// Activation boxes of a stage sit 2304 bytes apart: 2048 for 16 rows of 128 bytes plus 256, so that
-// consecutive boxes start two rows further into the 128-byte swizzle pattern (the pattern is tied to
-// the shared-memory address, chunk ^= (address / 128) % 8).  Lanes t and t + 2 of a warp read the same
-// chunk index of consecutive boxes; the shift sends them to different banks.
-constexpr int kXBoxPitch = 2304;
+// Activation boxes of a stage sit (slots * 128 + 256) bytes apart: the box itself plus two rows, so
+// that consecutive boxes start two rows further into the 128-byte swizzle pattern (the pattern is tied
+// to the shared-memory address, chunk ^= (address / 128) % 8).  Lanes t and t + 2 of a warp read the
+// same chunk index of consecutive boxes; the shift sends them to different banks.
+__host__ __device__ constexpr int x_box_pitch(int slots) { return slots * 128 + 256; }
 
 // Byte offset, inside a stage's activation area, of 16-byte chunk c (k = 8 c .. 8 c + 7 of the step)
 // of batch slot `slot`.
+template <int SLOTS>
 __device__ __forceinline__ uint32_t x_chunk_offset(int c, int slot) {
+    constexpr int PITCH = x_box_pitch(SLOTS);
     const int sb = c >> 3, cc = c & 7;
-    return (uint32_t)(sb * kXBoxPitch + slot * 128 + ((cc ^ ((slot + 2 * sb) & 7)) << 4));
+    return (uint32_t)(sb * PITCH + slot * 128 + ((cc ^ ((slot + 2 * sb) & 7)) << 4));
 }
 
 struct StreamArgs {
@@ -129,7 +134,7 @@ struct StreamArgs {
     const uint8_t *zeros;     // low-bit only
     void *Y;
     float *partial;           // [ctas][2][16 slots][128 features] fp32
-    int32_t *counters;        // [feature groups], zero on entry and on exit
+    int32_t *counters;        // [feature groups][kCounterStride], zero on entry and on exit
     int32_t *status;
     int M, coff, N, K, g_size;
     int g_shift;              // log2(g_size) when it is a power of two, else -1
@@ -154,12 +159,14 @@ template <int BITS, int NT, int GS>
 struct StreamCfg {
     using G = StepGeom<BITS>;
     static constexpr int SLOTS = NT * 8;
-    static constexpr int X_STAGE = ((G::X_BOXES * kXBoxPitch + 1023) / 1024) * 1024;
+    static constexpr int X_PITCH = x_box_pitch(SLOTS);
+    static constexpr int X_STAGE = ((G::X_BOXES * X_PITCH + 1023) / 1024) * 1024;
     static constexpr int X_TX = G::X_BOXES * SLOTS * 128;  // bytes the activation boxes deliver
     static constexpr int STAGE = kStepBytes + X_STAGE;
-    static constexpr int D_RAW = (kStageBudget * 1024) / STAGE;
+    static constexpr int D_RAW = (stage_budget_kb(NT) * 1024) / STAGE;
     static constexpr int D = D_RAW > kMaxStages ? kMaxStages : D_RAW;
-    static constexpr int SCRATCH = SLOTS * kTileRows * 4;
+    static constexpr int SUM_FLOATS = SLOTS * kTileRows;     // the sums k half 1 parks for k half 0
+    static constexpr int SCRATCH = 2 * SUM_FLOATS * 4;       // two parking buffers, used in turn
     static constexpr int SZ_OFF = D * STAGE + SCRATCH;
     static constexpr int SZ_WARP = 2 * 16 * kR * GS * 4;  // per consumer warp: two slots of (scale, zero) entries
     static constexpr int BAR_OFF = SZ_OFF + kConsumerWarps * SZ_WARP;
@@ -190,7 +197,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
     auto full_bar = [&](int d) { return bar0 + 8u * d; };
     auto empty_bar = [&](int d) { return bar0 + 128u + 8u * d; };
     const uint32_t cons_bar = bar0 + 256u;
-    volatile int32_t *flag = reinterpret_cast<volatile int32_t *>(base_ptr + Cfg::BAR_OFF + 320);
+    auto pub_bar = [&](int e) { return bar0 + 264u + 8u * e; };    // k half 0 warps -> publishing lane
+    auto role_bar = [&](int e) { return bar0 + 280u + 8u * e; };   // publishing lane -> consumer warps
+    volatile int32_t *is_last = reinterpret_cast<volatile int32_t *>(base_ptr + Cfg::BAR_OFF + 320);
 
     const int ctas = gridDim.x, cta = blockIdx.x;
     const int SPG = a.steps_per_group;
@@ -228,6 +237,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
             mbar_init(empty_bar(d), kConsumerWarps);
         }
         mbar_init(cons_bar, kConsumerWarps);
+        for (int e = 0; e < 2; ++e) {
+            mbar_init(pub_bar(e), kRowBlocks);
+            mbar_init(role_bar(e), 1);
+        }
         fence_barrier_init();
         prefetch_tensor_map(&wmap);
         prefetch_tensor_map(&xmap);
@@ -268,8 +281,56 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                 // activations of this k range: one [slots x 64] box per 64 k, rows past M read as zero
 #pragma unroll
                 for (int sb = 0; sb < Geo::X_BOXES; ++sb)
-                    tma_load_2d(x_stage(d) + sb * kXBoxPitch, &xmap, full_bar(d), ks * Geo::STEP_K + sb * 64, 0);
+                    tma_load_2d(x_stage(d) + sb * Cfg::X_PITCH, &xmap, full_bar(d), ks * Geo::STEP_K + sb * 64, 0);
             }
+        }
+        return;
+    }
+
+    // CTAs that hold steps of feature group rg_: the first and the last of them
+    auto sharers = [&](int rg_, int &c_first, int &c_last) {
+        const long long s_first = (long long)rg_ * SPG, s_last = s_first + SPG - 1;
+        c_first = (int)(((s_first + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
+        c_last = (int)(((s_last + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
+    };
+
+    if (warp == kPublishWarp) {
+        // ======================= publishing lane =======================
+        // A CTA has at most two parts of shared feature groups: the tail group (taken first) and the
+        // group its range starts in.  For each, once k half 0 has stored the part, this lane makes it
+        // visible, counts the CTA in and tells the consumers whether they were the last to arrive.  The
+        // consumers go on with their next steps meanwhile and only look at the answer at the end.
+        pdl_wait();
+        const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
+        if (rows <= 0 || lane != 0) return;
+        const int stop = n_tail > 0 ? rg_last * SPG : end;  // end of the part that starts at `beg`
+        const bool head_shared = ks_first > 0 || stop < (rg_first + 1) * SPG;
+        const int n_ev = (n_tail > 0 ? 1 : 0) + (head_shared ? 1 : 0);
+        const int rg0 = n_tail > 0 ? rg_last : rg_first, rg1 = rg_first;
+        // Both counts are issued before either answer is looked at, so that their round trips to
+        // the L2 overlap with each other and with the wait for the second part.
+        int old0 = 0, old1 = 0;
+        if (n_ev > 0) {
+            if (!mbar_wait(pub_bar(0), 0u, a.status)) return;
+            fence_acq_rel_gpu();  // the part stored by the k half 0 warps becomes visible before the count
+            old0 = atomicAdd(a.counters + (size_t)rg0 * kCounterStride, 1);
+        }
+        if (n_ev > 1) {
+            if (!mbar_wait(pub_bar(1), 0u, a.status)) return;
+            fence_acq_rel_gpu();
+            old1 = atomicAdd(a.counters + (size_t)rg1 * kCounterStride, 1);
+        }
+        for (int e = 0; e < n_ev; ++e) {
+            const int rg = e == 0 ? rg0 : rg1;
+            int c_first, c_last;
+            sharers(rg, c_first, c_last);
+            const bool last = (e == 0 ? old0 : old1) == c_last - c_first;
+            if (last) {
+                fence_acq_rel_gpu();       // the other CTAs' parts are visible to this CTA's loads from here on
+                a.counters[(size_t)rg * kCounterStride] = 0;        // every sharer has counted in: ready for the next call
+            }
+            is_last[e] = last ? 1 : 0;
+            mbar_arrive(role_bar(e));
         }
         return;
     }
@@ -310,7 +371,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                 if (BITS == 4) c = GS == 1 ? kh * 16 + t * 4 + i4 : kh * 16 + sg * 8 + t * 2 + i4;
                 else if (BITS == 8) c = kh * 8 + t * 2 + i4;
                 else c = kh * 4 + t;
-                x_off[nt][sg][i4] = x_chunk_offset(c, nt * 8 + g);
+                x_off[nt][sg][i4] = x_chunk_offset<SLOTS>(c, nt * 8 + g);
             }
 
     float acc[R][NT][4], accg[R][NT][4];
@@ -360,7 +421,15 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
 
     uint32_t cons_phase = 0;
     int first_ks = -1;  // k step at which this CTA entered the current feature group
+    int n_flush = 0, n_shared = 0, shared_rg0 = 0, shared_rg1 = 0;  // flushes so far; parts of shared groups so far
     Cursor cur = cursor_start();
+    auto store_y = [&](int n_base, int o, float v) {  // o = slot * 128 + feature within the group
+        const int slot = o / kTileRows, n = n_base + o % kTileRows;
+        if (slot >= rows || n >= a.N) return;
+        const int row = a.idx ? a.idx[slot] : slot;
+        if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
+        else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
+    };
 
     auto do_step = [&](int i) -> bool {
         const int d = i % D;
@@ -540,10 +609,16 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
             }
         }
 
-        // ---- end of this CTA's part of the feature group: combine and write ----
+        // ---- end of this CTA's part of the feature group: combine the k halves and write ----
         if (ks == SPG - 1 || end_of_part(i)) {
             const bool complete = first_ks == 0 && ks == SPG - 1;
-            // k half 1 parks its sums, k half 0 adds them (fixed order) and parks the total
+            if (!complete && n_shared >= 2) {  // cannot happen: a range has one tail and one head part
+                if (a.status) atomicExch(a.status, (int32_t)DMR_ERR_TIMEOUT);  // reported like a wait that ran out
+                return false;
+            }
+            // k half 1 parks its sums (two buffers in turn: the next flush's parking cannot overtake
+            // this flush's reading, there is a barrier between them), k half 0 adds them to its own
+            float *park = scratch + (n_flush & 1) * Cfg::SUM_FLOATS;
             if (kh == 1) {
 #pragma unroll
                 for (int r = 0; r < R; ++r)
@@ -551,91 +626,36 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
-                            scratch[(nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 16 * R + r * 16 + trow + 8 * (c >> 1)] = acc[r][nt][c];
+                            park[(nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 16 * R + r * 16 + trow + 8 * (c >> 1)] = acc[r][nt][c];
             }
             if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
             if (kh == 0) {
+                // and writes the outputs (group owned alone) or this CTA's part of a shared group
+                const int which = beg > rg * SPG ? 0 : 1;
+                float *mine = a.partial + ((size_t)cta * 2 + which) * (16 * kTileRows);
 #pragma unroll
                 for (int r = 0; r < R; ++r)
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
-                            float *p = scratch + (nt * 8 + 2 * t + (c & 1)) * kTileRows + rb * 16 * R + r * 16 + trow + 8 * (c >> 1);
-                            *p = acc[r][nt][c] + *p;
+                            const int slot = nt * 8 + 2 * t + (c & 1), f = rb * 16 * R + r * 16 + trow + 8 * (c >> 1);
+                            const float v = acc[r][nt][c] + park[slot * kTileRows + f];
+                            if (slot >= rows) continue;
+                            if (complete) store_y(rg * kTileRows, slot * kTileRows + f, v);
+                            else mine[slot * kTileRows + f] = v;
                         }
-            }
-            if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
-            const int n_base = rg * kTileRows;
-            auto store_y = [&](int o, float v) {
-                const int slot = o / kTileRows, n = n_base + o % kTileRows;
-                if (slot >= rows || n >= a.N) return;
-                const int row = a.idx ? a.idx[slot] : slot;
-                if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
-                else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
-            };
-            if (complete) {
-                for (int o = threadIdx.x; o < SLOTS * kTileRows; o += kConsumerWarps * 32) store_y(o, scratch[o]);
-            } else {
-                // Shared feature group: the CTA that arrives last adds all parts in CTA order and writes
-                // the result.  A CTA that finds every other part already published is that CTA and
-                // keeps its own part in shared memory; otherwise it publishes its part and counts in.
-                const int which = beg > rg * SPG ? 0 : 1;
-                const long long s_first = (long long)rg * SPG, s_last = s_first + SPG - 1;
-                const int c_first = (int)(((s_first + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
-                const int c_last = (int)(((s_last + 1) * ctas + a.total_steps - 1) / a.total_steps) - 1;
-                if (threadIdx.x == 0) {
-                    int seen;
-                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(a.counters + rg) : "memory");
-                    *flag = seen == c_last - c_first ? 2 : 0;
-                }
-                if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
-                int role = *flag;  // 2: reduce with the own part still in shared memory
-                if (role == 0) {
-                    float4 *mine = reinterpret_cast<float4 *>(a.partial + ((size_t)cta * 2 + which) * (16 * kTileRows));
-                    for (int o4 = threadIdx.x; o4 < SLOTS * kTileRows / 4; o4 += kConsumerWarps * 32)
-                        mine[o4] = reinterpret_cast<const float4 *>(scratch)[o4];
-                    if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
-                    if (threadIdx.x == 0) {
-                        __threadfence();  // the parts stored by the whole CTA before the barrier become visible first
-                        const int old = atomicAdd(a.counters + rg, 1);
-                        __threadfence();
-                        *flag = old == c_last - c_first ? 1 : 0;
-                    }
-                    if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
-                    role = *flag;  // 1: reduce from the published parts
-                }
-                if (role != 0) {
-                    // loads of up to eight parts are in flight together; the additions keep CTA order
-                    for (int o4 = threadIdx.x; o4 < SLOTS * kTileRows / 4; o4 += kConsumerWarps * 32) {
-                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (int cj0 = c_first; cj0 <= c_last; cj0 += 8) {
-                            float4 p[8];
-#pragma unroll
-                            for (int u = 0; u < 8; ++u) {
-                                const int cj = min(cj0 + u, c_last);
-                                const int wj = range_begin(cj, ctas, a.total_steps) > s_first ? 0 : 1;
-                                if (role == 2 && cj == cta) p[u] = reinterpret_cast<const float4 *>(scratch)[o4];
-                                else p[u] = __ldcg(reinterpret_cast<const float4 *>(a.partial + ((size_t)cj * 2 + wj) * (16 * kTileRows)) + o4);
-                            }
-#pragma unroll
-                            for (int u = 0; u < 8; ++u)
-                                if (cj0 + u <= c_last) {
-                                    v.x += p[u].x;
-                                    v.y += p[u].y;
-                                    v.z += p[u].z;
-                                    v.w += p[u].w;
-                                }
-                        }
-                        store_y(4 * o4 + 0, v.x);
-                        store_y(4 * o4 + 1, v.y);
-                        store_y(4 * o4 + 2, v.z);
-                        store_y(4 * o4 + 3, v.w);
-                    }
-                    if (threadIdx.x == 0) a.counters[rg] = 0;  // leave the counter ready for the next call
+                if (!complete) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(pub_bar(n_shared));
                 }
             }
-            if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;  // scratch and flag are free again
+            if (!complete) {
+                if (n_shared == 0) shared_rg0 = rg;
+                else shared_rg1 = rg;
+                ++n_shared;
+            }
+            ++n_flush;
 #pragma unroll
             for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -647,7 +667,44 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         return true;
     };
     for (int i = 0; i < nsteps; ++i)
-        if (!do_step(i)) break;
+        if (!do_step(i)) return;
+
+    // ---- shared feature groups this CTA was the last to count into: add all parts in CTA order ----
+    const int nvalid4 = rows * (kTileRows / 4);  // float4 items of the rows in use (slot-major)
+    for (int e = 0; e < n_shared; ++e) {
+        if (!mbar_wait(role_bar(e), 0u, a.status)) return;
+        if (is_last[e] == 0) continue;
+        const int rg = e == 0 ? shared_rg0 : shared_rg1;
+        int c_first, c_last;
+        sharers(rg, c_first, c_last);
+        const long long s_first = (long long)rg * SPG;
+        // loads of up to sixteen parts are in flight together; the additions keep CTA order
+        constexpr int PF = NT == 1 ? 12 : 8;
+        for (int o4 = threadIdx.x; o4 < nvalid4; o4 += kConsumerWarps * 32) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int cj0 = c_first; cj0 <= c_last; cj0 += PF) {
+                float4 p[PF];
+#pragma unroll
+                for (int u = 0; u < PF; ++u) {
+                    const int cj = min(cj0 + u, c_last);
+                    const int wj = range_begin(cj, ctas, a.total_steps) > s_first ? 0 : 1;
+                    p[u] = __ldcg(reinterpret_cast<const float4 *>(a.partial + ((size_t)cj * 2 + wj) * (16 * kTileRows)) + o4);
+                }
+#pragma unroll
+                for (int u = 0; u < PF; ++u)
+                    if (cj0 + u <= c_last) {
+                        v.x += p[u].x;
+                        v.y += p[u].y;
+                        v.z += p[u].z;
+                        v.w += p[u].w;
+                    }
+            }
+            store_y(rg * kTileRows, 4 * o4 + 0, v.x);
+            store_y(rg * kTileRows, 4 * o4 + 1, v.y);
+            store_y(rg * kTileRows, 4 * o4 + 2, v.z);
+            store_y(rg * kTileRows, 4 * o4 + 3, v.w);
+        }
+    }
 }
 
 int current_device() {
@@ -681,6 +738,9 @@ template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
 dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, const StreamArgs &a, int ctas,
                              cudaStream_t st) {
     using Cfg = StreamCfg<BITS, NT, GS>;
+    // 227 KB per CTA at most; two resident CTAs must fit into the SM's 228 KB with 1 KB reserved each
+    static_assert(Cfg::SMEM <= (NT == 1 ? (228 * 1024 - 2 * 1024) / 2 : 227 * 1024), "stage ring too large");
+    static_assert(Cfg::D >= 3, "stage ring too shallow");
     auto kernel = decode_stream_kernel<BITS, NT, GS, CE, OUT_F32>;
     static bool configured_on[64] = {};
     bool &configured = configured_on[current_device()];
@@ -726,7 +786,7 @@ dmr_status_t launch_stream_nt(const CUtensorMap &wmap, const CUtensorMap &xmap, 
 
 size_t stream_scratch_bytes(int N) {
     const size_t groups = (size_t)(N + kTileRows - 1) / kTileRows;
-    return round_up(groups * sizeof(int32_t), 256) + (size_t)kMaxStreamCtas * 2 * 16 * kTileRows * sizeof(float);
+    return groups * kCounterStride * sizeof(int32_t) + (size_t)kMaxStreamCtas * 2 * 16 * kTileRows * sizeof(float);
 }
 
 bool stream_supported(int M, int N, int K, int bits /*16 = bf16 weights*/, int g) {
@@ -750,7 +810,7 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     a.Y = Y;
     const size_t groups = (size_t)(N + kTileRows - 1) / kTileRows;
     a.counters = reinterpret_cast<int32_t *>(scratch);
-    a.partial = reinterpret_cast<float *>(reinterpret_cast<char *>(scratch) + round_up(groups * sizeof(int32_t), 256));
+    a.partial = reinterpret_cast<float *>(reinterpret_cast<char *>(scratch) + groups * kCounterStride * sizeof(int32_t));
     a.status = status;
     a.M = M;
     a.coff = sel.offset;
