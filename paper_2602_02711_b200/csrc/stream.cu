@@ -4,22 +4,29 @@
 // "Evaluation protocol", discussion of output length; App. "Latency coefficients").
 //
 // Work decomposition.  The weight matrix is cut into steps of [128 features x 128 bytes] (256
-// 4-bit codes, 128 8-bit codes or 64 bf16 weights per feature).  Steps are numbered feature-group
-// major, k minor, and CTA c of the persistent grid (one or two CTAs per SM) takes the contiguous range
-// [c * total / ctas, (c + 1) * total / ctas): every SM streams the same number of bytes whatever
-// the shape.  A feature group whose steps are shared by several CTAs is finished by the last of
-// them to arrive, which adds the partial sums in CTA order (no floating-point atomics), so the
-// summation order of an output depends on (N, K) and the SM count only - never on M, on the
-// row's position in the batch or on the other rows.  Counting a CTA into a shared group costs two
-// round trips to the L2 (fence, atomic); one lane of a warp of its own does that while the consumer
-// warps go on with their next steps, and the sums of the groups a CTA was last for are formed at
-// the end of the kernel by all consumer warps.
+// 4-bit codes, 128 8-bit codes or 64 bf16 weights per feature), numbered feature-group major, k
+// minor.  Two ways of dealing the steps out, chosen from the shape alone:
+//  - Large layers: CTA c of the persistent grid (one or two CTAs per SM) takes the contiguous range
+//    [c * total / ctas, (c + 1) * total / ctas), so every SM streams the same number of bytes whatever
+//    the shape.  A feature group whose steps are shared by several CTAs is finished by the last of
+//    them to arrive, which adds the partial sums in CTA order.  Counting a CTA into a shared group is
+//    a round trip to the L2; one lane of a warp of its own does that while the consumer warps go on
+//    with their next steps, and the sums of the groups a CTA was last for are formed at the end of the
+//    kernel by all consumer warps.
+//  - Small layers (up to 16 MB of codes, up to 8 rows), where that sum across CTAs is most of the run
+//    time: thread-block clusters of eight CTAs.  A cluster owns whole feature groups, rank r streams
+//    the r-th eighth of their k range, and at the end the cluster adds the eight sums of every output
+//    in rank order through distributed shared memory, each CTA taking an eighth of the outputs.
+// Either way there are no floating-point atomics, and the summation order of an output depends on
+// (N, K), the device and whether the batch has up to 8 or up to 16 rows - never on the row's
+// position in the batch or on the other rows.
 //
 // Inside a CTA one producer lane keeps a ring of stages full by TMA (cp.async.bulk.tensor,
 // 128-byte swizzle): the weight box and the matching activation boxes, all completing on the
 // stage's mbarrier (a routed batch is gathered into consecutive rows beforehand).  Eight consumer
-// warps each own 32 features and one half of the step's k range; the product runs on the tensor cores with the weights as the 16-row operand of mma.m16n8k16 and up
-// to 8 (or 2 x 8) activation rows as the 8-column operand.  4-bit codes are unpacked with one
+// warps each own 32 features and one half of the step's k range; the product runs on the tensor
+// cores with the weights as the 16-row operand of mma.m16n8k16 and up to 8 (or 2 x 8) activation
+// rows as the 8-column operand.  4-bit codes are unpacked with one
 // LOP3 per two codes ((w >> 4p) & 0x000F000F | 0x43004300 = {128 + q_p, 128 + q_{p+4}} as two
 // bf16) and one packed subtract of (128 + zero): the tensor-core operand is the exact integer
 // q - zero.  Products are accumulated per quantization group in fp32 and the group's scale is
@@ -47,6 +54,8 @@ constexpr int kStreamThreads = (kConsumerWarps + 2) * 32;  // + one producer war
 constexpr int kTileRows = 128;                              // features per step
 constexpr int kStepBytes = kTileRows * 128;                 // weight bytes per step (16 KB)
 constexpr int kMaxStages = 12;
+constexpr int kClusterSize = 8;                            // CTAs that share the k range of a feature group
+constexpr int kClusterMaxSteps = 1024;                     // layers of up to this many steps (16 MB) run in cluster mode
 // Shared memory for the stage ring, KB: two 8-row CTAs share an SM, a 16-row CTA has it alone.
 __host__ __device__ constexpr int stage_budget_kb(int nt) { return nt == 1 ? 92 : 100; }
 
@@ -95,7 +104,14 @@ __device__ __forceinline__ uint2 lds64(uint32_t addr) {
     return v;
 }
 
-__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+// Release: the parts this CTA stored (ordered before this lane by the barrier it waited on) are
+// visible to whoever reads the new count.  Acquire: if this was the last count, the other CTAs'
+// parts are visible to this CTA's loads that follow.
+__device__ __forceinline__ int atom_add_acq_rel(int32_t *p, int v) {
+    int old;
+    asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -140,10 +156,64 @@ struct StreamArgs {
     int g_shift;              // log2(g_size) when it is a power of two, else -1
     int steps_per_group;      // ceil(K / STEP_K)
     int total_steps;          // feature groups * steps_per_group
+    int part_groups;          // cluster mode: feature groups whose sums fit into a CTA's shared memory at once
 };
 
 __device__ __forceinline__ long long range_begin(int c, int ctas, int total) {
     return ((long long)c * total) / ctas;
+}
+
+// ---- thread-block clusters: rank, remote shared-memory addresses, remote barrier arrivals ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_count_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
+    return r;
+}
+// All threads of all CTAs of the cluster (hardware barrier; used once, after the barriers are set up).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of this CTA's shared-memory location `addr` in the CTA of rank `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_map(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Bounded wait that also orders the other CTAs' shared-memory writes before this thread's reads.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, int32_t *status) {
+    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (i > 128) __nanosleep(64);
+    }
+    if (status) atomicExch(status, (int32_t)DMR_ERR_TIMEOUT);
+    return false;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr));
+    return v;
 }
 
 // Consumer-warp barrier on an mbarrier (one arrival per warp) so that the wait is bounded.
@@ -166,7 +236,10 @@ struct StreamCfg {
     static constexpr int D_RAW = (stage_budget_kb(NT) * 1024) / STAGE;
     static constexpr int D = D_RAW > kMaxStages ? kMaxStages : D_RAW;
     static constexpr int SUM_FLOATS = SLOTS * kTileRows;     // the sums k half 1 parks for k half 0
-    static constexpr int SCRATCH = 2 * SUM_FLOATS * 4;       // two parking buffers, used in turn
+    // cluster mode keeps the sums of several feature groups here until the cluster adds them up
+    static constexpr int PART_BYTES = NT == 1 ? (BITS == 16 ? 16 : 20) * 1024 : 64 * 1024;
+    static constexpr int PARK_BYTES = 2 * SUM_FLOATS * 4;    // two parking buffers, used in turn
+    static constexpr int SCRATCH = PART_BYTES > PARK_BYTES ? PART_BYTES : PARK_BYTES;
     static constexpr int SZ_OFF = D * STAGE + SCRATCH;
     static constexpr int SZ_WARP = 2 * 16 * kR * GS * 4;  // per consumer warp: two slots of (scale, zero) entries
     static constexpr int BAR_OFF = SZ_OFF + kConsumerWarps * SZ_WARP;
@@ -176,7 +249,10 @@ struct StreamCfg {
 // BITS: 4 / 8 = packed codes, 16 = bf16 weights.  NT: 8-row activation tiles (1 or 2).
 // GS: quantization groups per 128-code unit (2 only for 4-bit codes with 64-wide groups).
 // CE: every unit a warp consumes ends its quantization group (group size == unit size).
-template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
+// CL: the CTAs of a thread-block cluster split the k range of the same feature groups and add their
+// sums through distributed shared memory (no trip through the L2); without it, CTAs take contiguous
+// step ranges and shared feature groups are summed through global memory by the last to arrive.
+template <int BITS, int NT, int GS, bool CE, bool OUT_F32, bool CL>
 __global__ void __launch_bounds__(kStreamThreads, NT == 1 ? 2 : 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ CUtensorMap xmap,
                      const StreamArgs a) {
@@ -200,36 +276,63 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
     auto pub_bar = [&](int e) { return bar0 + 264u + 8u * e; };    // k half 0 warps -> publishing lane
     auto role_bar = [&](int e) { return bar0 + 280u + 8u * e; };   // publishing lane -> consumer warps
     volatile int32_t *is_last = reinterpret_cast<volatile int32_t *>(base_ptr + Cfg::BAR_OFF + 320);
+    const uint32_t cl_full_bar = bar0 + 296u;   // cluster mode: every CTA's sums of the round are in place
+    const uint32_t cl_done_bar = bar0 + 304u;   // cluster mode: every CTA has finished reading the others' sums
 
     const int ctas = gridDim.x, cta = blockIdx.x;
     const int SPG = a.steps_per_group;
-    const int beg = (int)range_begin(cta, ctas, a.total_steps);
-    const int end = (int)range_begin(cta + 1, ctas, a.total_steps);
-    const int nsteps = end - beg;
     const int G = LOWBIT ? a.K / a.g_size : 1;
     // quantization group of input feature k without a division in the common cases
     auto group_of_k = [&](int k) { return a.g_shift >= 0 ? (k >> a.g_shift) : (G == 1 ? 0 : k / a.g_size); };
-    const int rg_first = beg / SPG, ks_first = beg - rg_first * SPG;
-    // Order of work.  A range that ends inside a feature group (shared with the next CTA) takes those
-    // last n_tail steps FIRST and then runs from its beginning up to that group: both CTAs of a shared
-    // group then produce their parts early and the fix-up hides behind the rest of the stream, and
-    // every CTA ends on a feature group it owns alone.
-    const int rg_last = (end - 1) / SPG;
-    const int n_tail = (end % SPG != 0 && rg_last > rg_first) ? end - rg_last * SPG : 0;
+    // ---- the work of this CTA ----
+    // Without clusters: the contiguous step range [beg, end).  A range that ends inside a feature group
+    // (shared with the next CTA) takes those last n_tail steps FIRST and then runs from its beginning up
+    // to that group: both CTAs of a shared group then produce their parts early and the fix-up hides
+    // behind the rest of the stream.
+    // With clusters: the feature groups [rg_first, g_end) of this cluster, and of each of them the k
+    // steps [ks_first, ks_end) of this CTA's rank.
+    int beg = 0, end = 0, nsteps = 0, rg_first = 0, ks_first = 0, rg_last = 0, n_tail = 0, g_end = 0, ks_end = 0;
+    uint32_t crank = 0;
+    if constexpr (CL) {
+        crank = cluster_ctarank();
+        const int groups = a.total_steps / SPG, nc = (int)cluster_count_x(), cid = (int)cluster_id_x();
+        rg_first = (int)(((long long)cid * groups) / nc);
+        g_end = (int)(((long long)(cid + 1) * groups) / nc);
+        ks_first = (int)crank * SPG / kClusterSize;
+        ks_end = ((int)crank + 1) * SPG / kClusterSize;
+        nsteps = (g_end - rg_first) * (ks_end - ks_first);
+    } else {
+        beg = (int)range_begin(cta, ctas, a.total_steps);
+        end = (int)range_begin(cta + 1, ctas, a.total_steps);
+        nsteps = end - beg;
+        rg_first = beg / SPG;
+        ks_first = beg - rg_first * SPG;
+        rg_last = (end - 1) / SPG;
+        n_tail = (end % SPG != 0 && rg_last > rg_first) ? end - rg_last * SPG : 0;
+    }
     struct Cursor {
         int rg, ks, i;
     };
     auto cursor_start = [&]() { return n_tail > 0 ? Cursor{rg_last, 0, 0} : Cursor{rg_first, ks_first, 0}; };
     auto cursor_next = [&](Cursor &c) {
-        if (++c.i == n_tail) {
-            c.rg = rg_first;
-            c.ks = ks_first;
-        } else if (++c.ks == SPG) {
-            c.ks = 0;
-            ++c.rg;
+        if constexpr (CL) {
+            ++c.i;
+            if (++c.ks == ks_end) {
+                c.ks = ks_first;
+                ++c.rg;
+            }
+        } else {
+            if (++c.i == n_tail) {
+                c.rg = rg_first;
+                c.ks = ks_first;
+            } else if (++c.ks == SPG) {
+                c.ks = 0;
+                ++c.rg;
+            }
         }
     };
-    auto end_of_part = [&](int i) { return i == n_tail - 1 || i == nsteps - 1; };
+    // step i (k step ks) is the last one this CTA has of its feature group
+    auto part_ends = [&](int i, int ks) { return CL ? ks == ks_end - 1 : (ks == SPG - 1 || i == n_tail - 1 || i == nsteps - 1); };
 
     if (threadIdx.x == 0) {
         for (int d = 0; d < D; ++d) {
@@ -241,11 +344,14 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
             mbar_init(pub_bar(e), kRowBlocks);
             mbar_init(role_bar(e), 1);
         }
+        mbar_init(cl_full_bar, kClusterSize);
+        mbar_init(cl_done_bar, kClusterSize);
         fence_barrier_init();
         prefetch_tensor_map(&wmap);
         prefetch_tensor_map(&xmap);
     }
     __syncthreads();
+    if constexpr (CL) cluster_sync_all();  // no CTA of the cluster is sent an arrival before its barriers exist
     pdl_launch_dependents();
 
     if (warp == kConsumerWarps) {
@@ -300,6 +406,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         // group its range starts in.  For each, once k half 0 has stored the part, this lane makes it
         // visible, counts the CTA in and tells the consumers whether they were the last to arrive.  The
         // consumers go on with their next steps meanwhile and only look at the answer at the end.
+        if constexpr (CL) return;
         pdl_wait();
         const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
         if (rows <= 0 || lane != 0) return;
@@ -308,27 +415,23 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         const int n_ev = (n_tail > 0 ? 1 : 0) + (head_shared ? 1 : 0);
         const int rg0 = n_tail > 0 ? rg_last : rg_first, rg1 = rg_first;
         // Both counts are issued before either answer is looked at, so that their round trips to
-        // the L2 overlap with each other and with the wait for the second part.
+        // the L2 overlap with each other and with the wait for the second part.  The count is one
+        // acquire-release atomic (measured faster than fence, atomic, fence).
         int old0 = 0, old1 = 0;
         if (n_ev > 0) {
             if (!mbar_wait(pub_bar(0), 0u, a.status)) return;
-            fence_acq_rel_gpu();  // the part stored by the k half 0 warps becomes visible before the count
-            old0 = atomicAdd(a.counters + (size_t)rg0 * kCounterStride, 1);
+            old0 = atom_add_acq_rel(a.counters + (size_t)rg0 * kCounterStride, 1);
         }
         if (n_ev > 1) {
             if (!mbar_wait(pub_bar(1), 0u, a.status)) return;
-            fence_acq_rel_gpu();
-            old1 = atomicAdd(a.counters + (size_t)rg1 * kCounterStride, 1);
+            old1 = atom_add_acq_rel(a.counters + (size_t)rg1 * kCounterStride, 1);
         }
         for (int e = 0; e < n_ev; ++e) {
             const int rg = e == 0 ? rg0 : rg1;
             int c_first, c_last;
             sharers(rg, c_first, c_last);
             const bool last = (e == 0 ? old0 : old1) == c_last - c_first;
-            if (last) {
-                fence_acq_rel_gpu();       // the other CTAs' parts are visible to this CTA's loads from here on
-                a.counters[(size_t)rg * kCounterStride] = 0;        // every sharer has counted in: ready for the next call
-            }
+            if (last) a.counters[(size_t)rg * kCounterStride] = 0;  // every sharer has counted in: ready for the next call
             is_last[e] = last ? 1 : 0;
             mbar_arrive(role_bar(e));
         }
@@ -572,8 +675,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                     // the group sum is complete for this warp when its next unit (one step further)
                     // lies in another group, in another feature group or outside this CTA's range
                     const int kpart = k0 + sg * (Geo::UNIT_K / GS);
-                    const bool closes = CE || group_of_k(kpart + Geo::STEP_K) != group_of_k(kpart) || ks == SPG - 1 ||
-                                        end_of_part(i) || kpart + Geo::STEP_K >= K;
+                    const bool closes = CE || group_of_k(kpart + Geo::STEP_K) != group_of_k(kpart) || part_ends(i, ks) ||
+                                        kpart + Geo::STEP_K >= K;
                     if (closes) {
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
@@ -610,7 +713,37 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         }
 
         // ---- end of this CTA's part of the feature group: combine the k halves and write ----
-        if (ks == SPG - 1 || end_of_part(i)) {
+        if constexpr (CL) {
+            if (part_ends(i, ks)) {
+                // the sums of both k halves go to this group's place in shared memory, where the
+                // cluster picks them up at the end of the round
+                float *dst = scratch + (size_t)((rg - rg_first) % a.part_groups) * a.M * kTileRows;
+                if (kh == 1) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const int slot = nt * 8 + 2 * t + (c & 1), f = rb * 16 * R + r * 16 + trow + 8 * (c >> 1);
+                                if (slot < a.M) dst[slot * kTileRows + f] = acc[r][nt][c];
+                            }
+                }
+                if (!consumer_sync(cons_bar, cons_phase, a.status)) return false;
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const int slot = nt * 8 + 2 * t + (c & 1), f = rb * 16 * R + r * 16 + trow + 8 * (c >> 1);
+                            if (kh == 0 && slot < a.M) dst[slot * kTileRows + f] += acc[r][nt][c];
+                            acc[r][nt][c] = 0.f;
+                        }
+            }
+            return true;
+        }
+        if (part_ends(i, ks)) {
             const bool complete = first_ks == 0 && ks == SPG - 1;
             if (!complete && n_shared >= 2) {  // cannot happen: a range has one tail and one head part
                 if (a.status) atomicExch(a.status, (int32_t)DMR_ERR_TIMEOUT);  // reported like a wait that ran out
@@ -666,6 +799,57 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         }
         return true;
     };
+    if constexpr (CL) {
+        // Rounds of up to part_groups feature groups: every CTA of the cluster streams its k slice of
+        // them, then the cluster adds the eight sums of every output in rank order, each CTA taking an
+        // eighth of the outputs and reading the others' shared memory directly.
+        const int my = ks_end - ks_first;
+        const uint32_t part_u32 = base + (uint32_t)(D * Cfg::STAGE);
+        uint32_t cl_phase = 0;
+        int i = 0;
+        for (int g0 = rg_first; g0 < g_end; g0 += a.part_groups) {
+            const int ng = min(a.part_groups, g_end - g0);
+            for (int s = 0; s < ng * my; ++s, ++i)
+                if (!do_step(i)) return;
+            if (!consumer_sync(cons_bar, cons_phase, a.status)) return;  // this CTA's sums are all in place
+            // lane q of the first warp tells CTA q (the eight arrivals travel side by side)
+            if (threadIdx.x < kClusterSize) mbar_arrive_remote(cluster_map(cl_full_bar, threadIdx.x));
+            if (!mbar_wait_cluster(cl_full_bar, cl_phase, a.status)) return;
+            const int per_group = rows * (kTileRows / 4);  // float4 items of one feature group
+            const int items = ng * per_group;
+            const int it0 = (int)crank * items / kClusterSize, it1 = ((int)crank + 1) * items / kClusterSize;
+            for (int it = it0 + (int)threadIdx.x; it < it1; it += kConsumerWarps * 32) {
+                const int gl = it / per_group, rem = it - gl * per_group;
+                const int slot = rem >> 5, f4 = rem & 31;
+                const uint32_t off = (uint32_t)(((gl * a.M + slot) * kTileRows + f4 * 4) * 4);
+                float4 p[kClusterSize];
+#pragma unroll
+                for (int q = 0; q < kClusterSize; ++q) {
+                    const bool has_steps = (q + 1) * SPG / kClusterSize > q * SPG / kClusterSize;
+                    p[q] = has_steps ? ld_cluster_f4(cluster_map(part_u32 + off, (uint32_t)q)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int q = 0; q < kClusterSize; ++q) {
+                    v.x += p[q].x;
+                    v.y += p[q].y;
+                    v.z += p[q].z;
+                    v.w += p[q].w;
+                }
+                const int n_base = (g0 + gl) * kTileRows, o = slot * kTileRows + f4 * 4;
+                store_y(n_base, o + 0, v.x);
+                store_y(n_base, o + 1, v.y);
+                store_y(n_base, o + 2, v.z);
+                store_y(n_base, o + 3, v.w);
+            }
+            // nobody may overwrite its sums (next round) or leave (last round) while others still read them
+            if (!consumer_sync(cons_bar, cons_phase, a.status)) return;
+            if (threadIdx.x < kClusterSize) mbar_arrive_remote(cluster_map(cl_done_bar, threadIdx.x));
+            if (!mbar_wait_cluster(cl_done_bar, cl_phase, a.status)) return;
+            cl_phase ^= 1u;
+        }
+        return;
+    }
     for (int i = 0; i < nsteps; ++i)
         if (!do_step(i)) return;
 
@@ -734,34 +918,86 @@ bool pdl_enabled() {
     return v != 0;
 }
 
-template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
-dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, const StreamArgs &a, int ctas,
-                             cudaStream_t st) {
+// Thread-block clusters are used unless the environment says DMR_CLUSTER=0.
+bool cluster_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("DMR_CLUSTER");
+        v = (e && e[0] == '0') ? 0 : 1;
+    }
+    return v != 0;
+}
+
+template <int BITS, int NT, int GS, bool CE, bool OUT_F32, bool CL>
+dmr_status_t launch_stream_cl(const CUtensorMap &wmap, const CUtensorMap &xmap, StreamArgs a, int ctas, cudaStream_t st,
+                              bool *unavailable) {
     using Cfg = StreamCfg<BITS, NT, GS>;
     // 227 KB per CTA at most; two resident CTAs must fit into the SM's 228 KB with 1 KB reserved each
     static_assert(Cfg::SMEM <= (NT == 1 ? (228 * 1024 - 2 * 1024) / 2 : 227 * 1024), "stage ring too large");
     static_assert(Cfg::D >= 3, "stage ring too shallow");
-    auto kernel = decode_stream_kernel<BITS, NT, GS, CE, OUT_F32>;
-    static bool configured_on[64] = {};
-    bool &configured = configured_on[current_device()];
-    if (!configured) {
+    auto kernel = decode_stream_kernel<BITS, NT, GS, CE, OUT_F32, CL>;
+    static int configured_on[64] = {};   // 0 = not yet, 1 = ready, -1 = cluster launch not possible on this device
+    static int max_clusters_on[64] = {};
+    const int dev = current_device();
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kStreamThreads, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (CL) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = kClusterSize;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
+    if (configured_on[dev] == 0) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM);
         if (e != cudaSuccess) {
             g_last_cuda_error = (int)e;
             return DMR_ERR_CUDA;
         }
-        configured = true;
+        configured_on[dev] = 1;
+        if (CL) {
+            // how many clusters of this kernel the device holds at once (a host-side query, no launch)
+            cfg.gridDim = dim3((unsigned)(kClusterSize * 64), 1, 1);
+            cfg.attrs = attr;
+            cfg.numAttrs = (unsigned)n_attr;
+            int n = 0;
+            e = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+            if (e != cudaSuccess || n < 1) {
+                (void)cudaGetLastError();
+                configured_on[dev] = -1;
+            } else {
+                max_clusters_on[dev] = n;
+            }
+        }
     }
-    cudaLaunchConfig_t cfg = {};
+    if (CL) {
+        if (configured_on[dev] < 0) {
+            *unavailable = true;
+            return DMR_OK;
+        }
+        const int groups = a.total_steps / a.steps_per_group;
+        int nc = max_clusters_on[dev];
+        if (nc * kClusterSize > kMaxStreamCtas) nc = kMaxStreamCtas / kClusterSize;
+        if (nc > groups) nc = groups;
+        ctas = nc * kClusterSize;
+        a.part_groups = (Cfg::PART_BYTES / 4) / (a.M * kTileRows);
+        if (a.part_groups < 1) {
+            *unavailable = true;
+            return DMR_OK;
+        }
+    }
     cfg.gridDim = dim3((unsigned)ctas, 1, 1);
-    cfg.blockDim = dim3(kStreamThreads, 1, 1);
-    cfg.dynamicSmemBytes = Cfg::SMEM;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    if (pdl_enabled()) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cfg.numAttrs = (unsigned)n_attr;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, wmap, xmap, a);
     if (e != cudaSuccess) {
         g_last_cuda_error = (int)e;
@@ -769,6 +1005,23 @@ dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, c
         return DMR_ERR_CUDA;
     }
     return check_launch();
+}
+
+// Cluster mode when the device can hold clusters of this kernel, else the global-memory fix-up.
+template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
+dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, const StreamArgs &a, int ctas,
+                             cudaStream_t st) {
+    // Clusters pay for small layers, where the sum across CTAs is most of the run time (measured: a
+    // 4096 x 4096 INT4 layer takes 6.5 us instead of 10.7).  Large layers keep the contiguous split: a
+    // cluster works on whole feature groups, which balances worse, and not every SM can hold its share
+    // of a cluster, which the longer streaming phase does not forgive.
+    if (cluster_enabled() && NT == 1 && a.total_steps <= kClusterMaxSteps) {
+        bool unavailable = false;
+        const dmr_status_t r = launch_stream_cl<BITS, NT, GS, CE, OUT_F32, true>(wmap, xmap, a, ctas, st, &unavailable);
+        if (!unavailable) return r;
+    }
+    bool unused = false;
+    return launch_stream_cl<BITS, NT, GS, CE, OUT_F32, false>(wmap, xmap, a, ctas, st, &unused);
 }
 
 template <int BITS, int GS, bool CE>
@@ -824,6 +1077,7 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     const long long total = (long long)groups * a.steps_per_group;
     if (total > 0x7FFFFFFF) return DMR_ERR_UNSUPPORTED;
     a.total_steps = (int)total;
+    a.part_groups = 0;
     int ctas = sm_count() * (M <= 8 ? 2 : 1);  // the 8-row kernels fit twice on an SM
     if (ctas > kMaxStreamCtas) ctas = kMaxStreamCtas;
     if (ctas > a.total_steps) ctas = a.total_steps;
