@@ -13,7 +13,7 @@
 //    a round trip to the L2; one lane of a warp of its own does that while the consumer warps go on
 //    with their next steps, and the sums of the groups a CTA was last for are formed at the end of the
 //    kernel by all consumer warps.
-//  - Small layers (up to 16 MB of codes, up to 8 rows), where that sum across CTAs is most of the run
+//  - Small layers (up to 25 MB of codes, up to 8 rows), where that sum across CTAs is most of the run
 //    time: thread-block clusters of eight CTAs.  A cluster owns whole feature groups, rank r streams
 //    the r-th eighth of their k range, and at the end the cluster adds the eight sums of every output
 //    in rank order through distributed shared memory, each CTA taking an eighth of the outputs.
@@ -55,7 +55,7 @@ constexpr int kTileRows = 128;                              // features per step
 constexpr int kStepBytes = kTileRows * 128;                 // weight bytes per step (16 KB)
 constexpr int kMaxStages = 12;
 constexpr int kClusterSize = 8;                            // CTAs that share the k range of a feature group
-constexpr int kClusterMaxSteps = 1024;                     // layers of up to this many steps (16 MB) run in cluster mode
+constexpr int kClusterMaxSteps = 1600;                     // layers of up to this many steps (25 MB) run in cluster mode
 // Shared memory for the stage ring, KB: two 8-row CTAs share an SM, a 16-row CTA has it alone.
 __host__ __device__ constexpr int stage_budget_kb(int nt) { return nt == 1 ? 92 : 100; }
 
@@ -983,6 +983,7 @@ dmr_status_t launch_stream_cl(const CUtensorMap &wmap, const CUtensorMap &xmap, 
         int nc = max_clusters_on[dev];
         if (nc * kClusterSize > kMaxStreamCtas) nc = kMaxStreamCtas / kClusterSize;
         if (nc > groups) nc = groups;
+        nc = (groups + (groups + nc - 1) / nc - 1) / ((groups + nc - 1) / nc);  // fewest clusters with the same longest share
         ctas = nc * kClusterSize;
         a.part_groups = (Cfg::PART_BYTES / 4) / (a.M * kTileRows);
         if (a.part_groups < 1) {
@@ -1011,8 +1012,8 @@ dmr_status_t launch_stream_cl(const CUtensorMap &wmap, const CUtensorMap &xmap, 
 template <int BITS, int NT, int GS, bool CE, bool OUT_F32>
 dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, const StreamArgs &a, int ctas,
                              cudaStream_t st) {
-    // Clusters pay for small layers, where the sum across CTAs is most of the run time (measured: a
-    // 4096 x 4096 INT4 layer takes 6.5 us instead of 10.7).  Large layers keep the contiguous split: a
+    // Clusters pay for small and medium layers, where the sum across CTAs is most of the run time
+    // (measured: a 4096 x 4096 INT4 layer takes 6.5 us instead of 10.7).  Large layers keep the contiguous split: a
     // cluster works on whole feature groups, which balances worse, and not every SM can hold its share
     // of a cluster, which the longer streaming phase does not forgive.
     if (cluster_enabled() && NT == 1 && a.total_steps <= kClusterMaxSteps) {
