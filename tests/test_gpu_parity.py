@@ -151,6 +151,19 @@ def test_lowbit_linear_shapes(M, N, K, bits, group):
     run_lowbit_case(M, N, K, bits, group, seed=3)
 
 
+@pytest.mark.parametrize("M,N,K,bits,group", [
+    (8, 22016, 2048, 4, 128),  # 172 feature groups over at most 33 clusters: more than fit into shared memory at once (two rounds)
+    (3, 4224, 768, 4, 128),    # 3 steps per feature group: five of the eight ranks of a cluster have no k slice
+    (7, 1000, 4096, 8, 128),   # INT8, ragged N: 8 feature groups, 8 clusters
+    (1, 4096, 4096, 4, 64),    # g = 64 (two groups per 128-code unit), one feature group per cluster
+    (8, 136, 11008, 4, 0),     # per-channel scales, 43 steps per group: uneven k slices (5 and 6 steps)
+])
+def test_lowbit_linear_cluster_mode_shapes(M, N, K, bits, group):
+    """Small layers with up to 8 rows: the CTAs of a thread-block cluster split each feature group's k
+    range and add their sums through distributed shared memory."""
+    run_lowbit_case(M, N, K, bits, group, seed=5)
+
+
 def test_prefill_accuracy_margin_and_extreme_ranges():
     # the prefill kernel multiplies fp16 operands after rescaling activation rows and weight scales by
     # powers of two: the error against the exact oracle stays well inside the 2e-3 bound ...
