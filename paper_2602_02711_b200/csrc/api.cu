@@ -155,7 +155,7 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
             Xc = ws.xg_stream;
         }
         dmr_status_t r = launch_stream(Xc, mc, s, qweight, scales, zeros, N, K, f.bits, g, Yc, out, ws.stream_scratch,
-                                       ws.status, st);
+                                       ws.status, st, M);
         if (r != DMR_OK) return r;
     }
     return DMR_OK;
@@ -191,7 +191,7 @@ dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, 
             if (rg != DMR_OK) return rg;
             Xc = ws.xg_stream;
         }
-        dmr_status_t r = launch_stream(Xc, mc, s, W, nullptr, nullptr, N, K, 16, K, Yc, out, ws.stream_scratch, ws.status, st);
+        dmr_status_t r = launch_stream(Xc, mc, s, W, nullptr, nullptr, N, K, 16, K, Yc, out, ws.stream_scratch, ws.status, st, M);
         if (r != DMR_OK) return r;
     }
     return DMR_OK;

@@ -13,13 +13,14 @@
 //    a round trip to the L2; one lane of a warp of its own does that while the consumer warps go on
 //    with their next steps, and the sums of the groups a CTA was last for are formed at the end of the
 //    kernel by all consumer warps.
-//  - Small layers (up to 25 MB of codes, up to 8 rows), where that sum across CTAs is most of the run
-//    time: thread-block clusters of eight CTAs.  A cluster owns whole feature groups, rank r streams
-//    the r-th eighth of their k range, and at the end the cluster adds the eight sums of every output
-//    in rank order through distributed shared memory, each CTA taking an eighth of the outputs.
+//  - Small layers (up to 25 MB of codes), where that sum across CTAs is most of the run time:
+//    thread-block clusters of eight CTAs (four for the 16-row kernels).  A cluster owns whole feature
+//    groups, rank r streams the r-th part of their k range, and at the end the cluster adds the sums
+//    of every output in rank order through distributed shared memory, each CTA taking its share of the
+//    outputs.
 // Either way there are no floating-point atomics, and the summation order of an output depends on
-// (N, K), the device and whether the batch has up to 8 or up to 16 rows - never on the row's
-// position in the batch or on the other rows.
+// (N, K), the device and whether the call has up to 8 rows or more - never on the row's position in
+// the batch or on the other rows (all chunks of a call with more than 16 rows use the 16-row kernel).
 //
 // Inside a CTA one producer lane keeps a ring of stages full by TMA (cp.async.bulk.tensor,
 // 128-byte swizzle): the weight box and the matching activation boxes, all completing on the
@@ -54,7 +55,9 @@ constexpr int kStreamThreads = (kConsumerWarps + 2) * 32;  // + one producer war
 constexpr int kTileRows = 128;                              // features per step
 constexpr int kStepBytes = kTileRows * 128;                 // weight bytes per step (16 KB)
 constexpr int kMaxStages = 12;
-constexpr int kClusterSize = 8;                            // CTAs that share the k range of a feature group
+// CTAs that share the k range of a feature group: 8 for the 8-row kernels (two CTAs per SM), 4 for the
+// 16-row kernels (one CTA per SM: clusters of 8 SMs would leave a fifth of the SMs without work).
+__host__ __device__ constexpr int cluster_size(int nt) { return nt == 1 ? 8 : 4; }
 constexpr int kClusterMaxSteps = 1600;                     // layers of up to this many steps (25 MB) run in cluster mode
 // Shared memory for the stage ring, KB: two 8-row CTAs share an SM, a 16-row CTA has it alone.
 __host__ __device__ constexpr int stage_budget_kb(int nt) { return nt == 1 ? 92 : 100; }
@@ -157,6 +160,7 @@ struct StreamArgs {
     int steps_per_group;      // ceil(K / STEP_K)
     int total_steps;          // feature groups * steps_per_group
     int part_groups;          // cluster mode: feature groups whose sums fit into a CTA's shared memory at once
+    int wide;                 // host side: 1 = the 16-row kernel (the call has more than 8 rows)
 };
 
 __device__ __forceinline__ long long range_begin(int c, int ctas, int total) {
@@ -259,6 +263,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
     using Cfg = StreamCfg<BITS, NT, GS>;
     using Geo = StepGeom<BITS>;
     constexpr int D = Cfg::D, SLOTS = Cfg::SLOTS, R = kR;
+    constexpr int kClusterSize = cluster_size(NT);
     constexpr bool LOWBIT = BITS != 16;
     constexpr int WPS = 4 / GS;  // 32-bit code words per lane, feature and group part
     extern __shared__ uint8_t smem_dyn[];
@@ -801,8 +806,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
     };
     if constexpr (CL) {
         // Rounds of up to part_groups feature groups: every CTA of the cluster streams its k slice of
-        // them, then the cluster adds the eight sums of every output in rank order, each CTA taking an
-        // eighth of the outputs and reading the others' shared memory directly.
+        // them, then the cluster adds the sums of every output in rank order, each CTA taking its share
+        // of the outputs and reading the others' shared memory directly.
         const int my = ks_end - ks_first;
         const uint32_t part_u32 = base + (uint32_t)(D * Cfg::STAGE);
         uint32_t cl_phase = 0;
@@ -812,7 +817,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
             for (int s = 0; s < ng * my; ++s, ++i)
                 if (!do_step(i)) return;
             if (!consumer_sync(cons_bar, cons_phase, a.status)) return;  // this CTA's sums are all in place
-            // lane q of the first warp tells CTA q (the eight arrivals travel side by side)
+            // lane q of the first warp tells CTA q (the arrivals travel side by side)
             if (threadIdx.x < kClusterSize) mbar_arrive_remote(cluster_map(cl_full_bar, threadIdx.x));
             if (!mbar_wait_cluster(cl_full_bar, cl_phase, a.status)) return;
             const int per_group = rows * (kTileRows / 4);  // float4 items of one feature group
@@ -932,6 +937,7 @@ template <int BITS, int NT, int GS, bool CE, bool OUT_F32, bool CL>
 dmr_status_t launch_stream_cl(const CUtensorMap &wmap, const CUtensorMap &xmap, StreamArgs a, int ctas, cudaStream_t st,
                               bool *unavailable) {
     using Cfg = StreamCfg<BITS, NT, GS>;
+    constexpr int kClusterSize = cluster_size(NT);
     // 227 KB per CTA at most; two resident CTAs must fit into the SM's 228 KB with 1 KB reserved each
     static_assert(Cfg::SMEM <= (NT == 1 ? (228 * 1024 - 2 * 1024) / 2 : 227 * 1024), "stage ring too large");
     static_assert(Cfg::D >= 3, "stage ring too shallow");
@@ -1016,7 +1022,7 @@ dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, c
     // (measured: a 4096 x 4096 INT4 layer takes 6.5 us instead of 10.7).  Large layers keep the contiguous split: a
     // cluster works on whole feature groups, which balances worse, and not every SM can hold its share
     // of a cluster, which the longer streaming phase does not forgive.
-    if (cluster_enabled() && NT == 1 && a.total_steps <= kClusterMaxSteps) {
+    if (cluster_enabled() && a.total_steps <= kClusterMaxSteps) {
         bool unavailable = false;
         const dmr_status_t r = launch_stream_cl<BITS, NT, GS, CE, OUT_F32, true>(wmap, xmap, a, ctas, st, &unavailable);
         if (!unavailable) return r;
@@ -1028,7 +1034,7 @@ dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, c
 template <int BITS, int GS, bool CE>
 dmr_status_t launch_stream_nt(const CUtensorMap &wmap, const CUtensorMap &xmap, const StreamArgs &a, int ctas,
                               dmr_out_t out, cudaStream_t st) {
-    if (a.M <= 8) {
+    if (!a.wide) {
         if (out == DMR_OUT_F32) return launch_stream_t<BITS, 1, GS, CE, true>(wmap, xmap, a, ctas, st);
         return launch_stream_t<BITS, 1, GS, CE, false>(wmap, xmap, a, ctas, st);
     }
@@ -1054,9 +1060,10 @@ bool stream_supported(int M, int N, int K, int bits /*16 = bf16 weights*/, int g
 
 dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,
                            const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
-                           void *scratch, int32_t *status, cudaStream_t st) {
+                           void *scratch, int32_t *status, cudaStream_t st, int batch_rows) {
     const int step_k = 1024 / bits;
     StreamArgs a;
+    a.wide = (batch_rows > M ? batch_rows : M) > 8 ? 1 : 0;
     a.idx = sel.idx;
     a.count = sel.count;
     a.scales = scales;
@@ -1079,7 +1086,7 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     if (total > 0x7FFFFFFF) return DMR_ERR_UNSUPPORTED;
     a.total_steps = (int)total;
     a.part_groups = 0;
-    int ctas = sm_count() * (M <= 8 ? 2 : 1);  // the 8-row kernels fit twice on an SM
+    int ctas = sm_count() * (a.wide ? 1 : 2);  // the 8-row kernels fit twice on an SM
     if (ctas > kMaxStreamCtas) ctas = kMaxStreamCtas;
     if (ctas > a.total_steps) ctas = a.total_steps;
     CUtensorMap wmap;
@@ -1090,7 +1097,7 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     // X holds M consecutive rows (for a routed call: the gathered rows); box = [8 or 16 slots][64 k]
     CUtensorMap xmap;
     if (!make_tensor_map_2d(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)K * 2,
-                            M <= 8 ? 8 : 16, 64, TmaSwizzle::k128B))
+                            a.wide ? 16 : 8, 64, TmaSwizzle::k128B))
         return DMR_ERR_CUDA;
     if (bits == 16) return launch_stream_nt<16, 1, false>(wmap, xmap, a, ctas, out, st);
     if (bits == 8) {

@@ -289,6 +289,15 @@ def test_routed_linear_int8_and_ragged():
     routed_case(23, 136, 384, 8, 0, mask)
 
 
+@pytest.mark.parametrize("M,N,K", [(24, 1000, 4096), (31, 4096, 1024), (20, 22016, 512)])
+def test_routed_rows_move_between_chunks(M, N, K):
+    """17 to 32 rows run as chunks of 16: a routed call moves rows from one chunk to another, and they must
+    still come out bit for bit as in the unrouted call (every chunk uses the same kernel and summation
+    order), on layers large enough for feature groups to be shared between CTAs or clusters."""
+    mask = inputs.precision_mask(M, 0.4, seed=M)
+    routed_case(M, N, K, 4, 128, mask)
+
+
 def test_routed_linear_prefill_sized_batch():
     # above 128 rows both the routed and the unrouted call take the persistent tensor-core kernel
     mask = inputs.precision_mask(300, 0.3, seed=15)
