@@ -167,6 +167,27 @@ dmr_status_t dmr_lowbit_linear_noalloc(const void *X_bf16, int M, const void *qw
                                        const void *zeros, int N, int K, dmr_qformat_t f, void *Y,
                                        dmr_out_t out, void *stream);
 
+/*
+ * Step-wise KL divergence between the high- and the low-precision model's action distributions,
+ * the signal the KL-ST router is trained on (Sec. "KL-ST Stage"; App. on search and click steps:
+ * KL_t = mean over the action tokens i of step t of KL(pi_high(x_i) || pi_low(x_i))).
+ *   logits_high, logits_low : device, [T][V] row-major, bf16 (dtype = DMR_OUT_BF16) or fp32
+ *                             (DMR_OUT_F32); row i holds the logits both models give for action
+ *                             token i.  16-byte aligned.  Read once, not modified.
+ *   step_offsets            : device, int32 [S + 1], non-decreasing, within [0, T]: step s owns the
+ *                             tokens [step_offsets[s], step_offsets[s + 1]).  May be NULL when S = 0.
+ *   kl_token                : device, fp32 [T], written: KL(softmax(high_i) || softmax(low_i)) in nats.
+ *   kl_step                 : device, fp32 [S], written: the mean of kl_token over the step's tokens
+ *                             (added in token order), 0 for a step without tokens.
+ * fp32 arithmetic, one pass over the logits; a vocabulary entry with probability 0 under the
+ * high-precision model (logit -inf) contributes nothing.  No workspace, no allocation.
+ * Errors: DMR_ERR_INVALID_ARG (null pointer, T < 0, V < 1, S < 0, bad dtype), DMR_ERR_ALIGNMENT,
+ * DMR_ERR_CUDA.  T = 0 writes only kl_step (zeros).  The caller owns all buffers.
+ */
+dmr_status_t dmr_stepwise_kl(const void *logits_high, const void *logits_low, dmr_out_t dtype, int T,
+                             int V, const int32_t *step_offsets, int S, float *kl_token, float *kl_step,
+                             void *stream);
+
 /* Reads the status word a previous call may have set in `workspace` (DMR_OK or DMR_ERR_TIMEOUT).
  * Synchronises `stream`. */
 dmr_status_t dmr_workspace_status(const void *workspace, void *stream);

@@ -199,3 +199,38 @@ def route_partition(mask):
     nl = ctypes.c_int32(0)
     _check(_L().oracle_route_partition(_p(mask), M, _p(ih), _p(il), ctypes.byref(nh), ctypes.byref(nl)))
     return ih[:nh.value].copy(), il[:nl.value].copy()
+
+
+def stepwise_kl(logits_high: np.ndarray, logits_low: np.ndarray, step_offsets):
+    """Step-wise KL divergence (Sec. "KL-ST Stage"; App. on search and click steps):
+    KL_t = mean over the action tokens i of step t of KL(pi_high(x_i) || pi_low(x_i)), pi = softmax(logits).
+
+    `logits_high`, `logits_low`: [T][V] arrays, uint16 (bf16 bit patterns) or floating point; everything is
+    computed in float64 from the definition: log-softmax of each row, p = exp(log-softmax of the high
+    row), KL = sum_v p_v (log p_v - log q_v) with the convention that p_v = 0 contributes 0.
+    `step_offsets`: S + 1 non-decreasing token indices. Returns (kl_step [S], kl_token [T]) in nats;
+    a step without tokens has KL 0.
+    """
+    def as_f64(a):
+        a = np.asarray(a)
+        if a.dtype == np.uint16:
+            return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        return a.astype(np.float64)
+
+    A, B = as_f64(logits_high), as_f64(logits_low)
+    T = A.shape[0]
+    kl_token = np.zeros(T, dtype=np.float64)
+    for i in range(T):
+        a, b = A[i], B[i]
+        log_p = a - (a.max() + np.log(np.sum(np.exp(a - a.max()))))
+        log_q = b - (b.max() + np.log(np.sum(np.exp(b - b.max()))))
+        p = np.exp(log_p)
+        with np.errstate(invalid="ignore"):
+            terms = np.where(p > 0.0, p * (log_p - log_q), 0.0)
+        kl_token[i] = np.sum(terms)
+    off = np.asarray(step_offsets, dtype=np.int64)
+    kl_step = np.zeros(max(len(off) - 1, 0), dtype=np.float64)
+    for s in range(len(kl_step)):
+        seg = kl_token[off[s]:off[s + 1]]
+        kl_step[s] = seg.mean() if len(seg) else 0.0
+    return kl_step, kl_token

@@ -55,6 +55,8 @@ def lib() -> ctypes.CDLL:
         getattr(L, name).argtypes = [i32, i32, QFormat]
     L.dmr_workspace_bytes.restype = sz
     L.dmr_workspace_bytes.argtypes = [i32, i32, i32, i32, QFormat]
+    L.dmr_stepwise_kl.restype = i32
+    L.dmr_stepwise_kl.argtypes = [vp, vp, i32, i32, i32, vp, i32, vp, vp, vp]
     L.dmr_quantize.restype = i32
     L.dmr_quantize.argtypes = [vp, i32, i32, QFormat, vp, vp, vp, vp, vp]
     L.dmr_dequantize.restype = i32
@@ -250,6 +252,27 @@ def dmr_lowbit_linear_host(X_host: torch.Tensor, q: QuantizedLinear, Y_host: tor
                                     _ptr(Y_host), out, _ptr(staging), staging.numel(), _ptr(workspace),
                                     workspace.numel(), _stream(stream)))
     return Y_host
+
+
+def dmr_stepwise_kl(logits_high: torch.Tensor, logits_low: torch.Tensor, step_offsets: torch.Tensor, stream=None):
+    """Step-wise KL divergence of two [T, V] logit tensors (bf16 or fp32, same dtype).
+
+    `step_offsets` is an int32 device tensor [S + 1]. Returns (kl_step [S], kl_token [T]), fp32.
+    """
+    if logits_high.dtype not in (torch.bfloat16, torch.float32) or logits_low.dtype != logits_high.dtype:
+        raise DmrError(1, "logits must both be bf16 or both be fp32")
+    a = _dev(logits_high, logits_high.dtype, "logits_high")
+    b = _dev(logits_low, logits_high.dtype, "logits_low")
+    if a.dim() != 2 or a.shape != b.shape:
+        raise DmrError(1, "logits must be [T, V] tensors of the same shape")
+    off = _dev(step_offsets, torch.int32, "step_offsets")
+    T, V = a.shape
+    S = off.numel() - 1
+    kl_token = torch.empty((T,), dtype=torch.float32, device=a.device)
+    kl_step = torch.empty((max(S, 0),), dtype=torch.float32, device=a.device)
+    dtype = OUT_F32 if a.dtype == torch.float32 else OUT_BF16
+    _check(lib().dmr_stepwise_kl(_ptr(a), _ptr(b), dtype, T, V, _ptr(off), S, _ptr(kl_token), _ptr(kl_step), _stream(stream)))
+    return kl_step, kl_token
 
 
 def dmr_lowbit_linear_noalloc(X: torch.Tensor, q: QuantizedLinear, Y: torch.Tensor, out: int = OUT_BF16, stream=None):

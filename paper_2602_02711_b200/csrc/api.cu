@@ -397,6 +397,18 @@ dmr_status_t dmr_lowbit_linear_host(const void *X_host, int M, const void *qweig
     return DMR_OK;
 }
 
+dmr_status_t dmr_stepwise_kl(const void *logits_high, const void *logits_low, dmr_out_t dtype, int T, int V,
+                             const int32_t *step_offsets, int S, float *kl_token, float *kl_step, void *stream) {
+    if (T < 0 || V < 1 || S < 0) return DMR_ERR_INVALID_ARG;
+    if (dtype != DMR_OUT_BF16 && dtype != DMR_OUT_F32) return DMR_ERR_INVALID_ARG;
+    if (T > 0 && (!logits_high || !logits_low || !kl_token)) return DMR_ERR_INVALID_ARG;
+    if (S > 0 && (!step_offsets || !kl_step)) return DMR_ERR_INVALID_ARG;
+    if (!aligned16(logits_high) || !aligned16(logits_low)) return DMR_ERR_ALIGNMENT;
+    if (T == 0 && S == 0) return DMR_OK;
+    return launch_stepwise_kl(logits_high, logits_low, dtype == DMR_OUT_F32, T, V, step_offsets, S, kl_token, kl_step,
+                              reinterpret_cast<cudaStream_t>(stream));
+}
+
 dmr_status_t dmr_workspace_status(const void *workspace, void *stream) {
     if (!workspace) return DMR_ERR_INVALID_ARG;
     int32_t v = 0;

@@ -116,4 +116,9 @@ dmr_status_t launch_simple_dense(const uint16_t *X, int M, RowSel sel, const uin
 dmr_status_t launch_route_partition(const uint8_t *mask, int M, int32_t *idx_high, int32_t *idx_low,
                                     int32_t *counts, cudaStream_t st);
 
+// Step-wise KL divergence: kl_token[i] = KL(softmax(high[i]) || softmax(low[i])) for T rows of V logits
+// (bf16 or fp32), kl_step[s] = mean of kl_token over [offsets[s], offsets[s + 1]).
+dmr_status_t launch_stepwise_kl(const void *high, const void *low, bool f32, int T, int V, const int32_t *offsets, int S,
+                                float *kl_token, float *kl_step, cudaStream_t st);
+
 }  // namespace dmr

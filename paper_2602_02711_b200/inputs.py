@@ -121,3 +121,33 @@ LAYER_32B = {
     "gate": (27648, 5120),
     "down": (5120, 27648),
 }
+
+
+TID_LOGIT = 71
+TID_LOGIT_NOISE = 72
+TID_STEP_LEN = 73
+
+
+def logit_pair(T: int, V: int, seed: int = 0, index: int = 0, critical_frac: float = 0.1):
+    """Two [T][V] float64 logit matrices standing in for the high- and the low-precision model on the
+    same action tokens: high ~ N(0, 2.5^2) with a few strongly preferred entries per token; low =
+    high + N(0, 0.1^2) for most tokens and + N(0, 1.5^2) for a `critical_frac` of them (most steps
+    agree closely, a few deviate a lot)."""
+    g = _rng(seed, TID_LOGIT, index)
+    high = g.standard_normal(size=(T, V), dtype=np.float64) * 2.5
+    for i in range(T):
+        top = g.integers(0, V, size=3)
+        high[i, top] += np.array([9.0, 7.0, 6.0])
+    gn = _rng(seed, TID_LOGIT_NOISE, index)
+    sigma = np.where(gn.random(T) < critical_frac, 1.5, 0.1)
+    low = high + gn.standard_normal(size=(T, V), dtype=np.float64) * sigma[:, None]
+    return high, low
+
+
+def step_offsets(T: int, mean_len: int = 12, seed: int = 0, index: int = 0) -> np.ndarray:
+    """int32 [S + 1] token offsets of consecutive steps whose action blocks have 0 .. 2 mean_len tokens."""
+    g = _rng(seed, TID_STEP_LEN, index)
+    offs = [0]
+    while offs[-1] < T:
+        offs.append(min(T, offs[-1] + int(g.integers(0, 2 * mean_len + 1))))
+    return np.asarray(offs, dtype=np.int32)
