@@ -220,7 +220,7 @@ def run_ours(args):
     peaks = load_peaks()
     fmt = QFormat(BITS, GROUP)
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost"}
+    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost", "kl"}
 
     def bf16_dev(bits_np):
         return torch.from_numpy(bits_np.view(np.int16)).view(torch.bfloat16).to(dev)
@@ -548,6 +548,21 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
                 del qs
         out["crossover_32b"] = cx
 
+    if "kl" in sections:
+        # Step-wise KL divergence: two [T][V] bf16 logit tensors (1.24 GB, far beyond the L2) read once.
+        T, V = 2048, 151936
+        g = torch.Generator(device=dev)
+        g.manual_seed(97)
+        hi = (torch.randn((T, V), generator=g, device=dev, dtype=torch.float32) * 2.5).to(torch.bfloat16)
+        lo = (hi.float() + torch.randn((T, V), generator=g, device=dev, dtype=torch.float32) * 0.1).to(torch.bfloat16)
+        offs = torch.from_numpy(inputs.step_offsets(T, 12, seed=3)).to(dev)
+        t = timeit(lambda: dmr.dmr_stepwise_kl(hi, lo, offs), reps=10, warm=3)
+        b = 2.0 * T * V * 2
+        out["stepwise_kl"] = {"us": t * 1e6, "gbs": b / t / 1e9, "frac_hbm": b / t / 1e9 / peaks["hbm_gbs"],
+                              "tokens_per_s": T / t,
+                              "workload": f"{T} action tokens x {V} logits, bf16, two models, {int(offs.numel()) - 1} steps"}
+        del hi, lo
+
     if "quantize" in sections:
         qz = {}
         for name, (N, K) in inputs.LAYER_7B.items():
@@ -565,7 +580,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost")
+    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost,kl")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
