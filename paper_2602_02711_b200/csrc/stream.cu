@@ -445,9 +445,6 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
     }
 
     // ======================= consumer warps =======================
-    pdl_wait();
-    const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
-    if (rows <= 0) return;
     const int rb = warp % kRowBlocks, kh = warp / kRowBlocks;  // feature block, k half
     const int g = lane >> 2, t = lane & 3;
     const int trow = tile_row_of(g);
@@ -516,17 +513,22 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
         }
         __syncwarp();
     };
-    uint32_t pend[GS][2];
+    // The scales and zero points of the first two steps are weights too: fetch them before waiting
+    // for the preceding kernel, so that their trip to DRAM is not on the path to the first step.
+    uint32_t pend[GS][2], first_sz[GS][2];
     Cursor pf = cursor_start();  // step the next fetch is for
     if (nsteps > 0) {
-        sz_fetch(pf.rg, pf.ks, pend);
-        sz_store(0, pend);
+        sz_fetch(pf.rg, pf.ks, first_sz);
         cursor_next(pf);
     }
     if (nsteps > 1) {
         sz_fetch(pf.rg, pf.ks, pend);
         cursor_next(pf);
     }
+    pdl_wait();
+    const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
+    if (rows <= 0) return;
+    if (nsteps > 0) sz_store(0, first_sz);
 
     uint32_t cons_phase = 0;
     int first_ks = -1;  // k step at which this CTA entered the current feature group
