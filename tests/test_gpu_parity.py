@@ -334,7 +334,7 @@ def test_lowbit_linear_host_matches_device_call():
 
 # ---------------- full-size shapes, sampled outputs ----------------
 
-@pytest.mark.parametrize("name,M", [("qkv", 1), ("o", 8), ("gate_up", 16), ("down", 16)])
+@pytest.mark.parametrize("name,M", [("qkv", 1), ("o", 8), ("gate_up", 16), ("down", 16), ("gate_up", 4)])
 def test_7b_decode_shapes_sampled(name, M):
     N, K = inputs.LAYER_7B[name]
     W = inputs.weights(N, K, seed=0, index=sorted(inputs.LAYER_7B).index(name))
