@@ -47,11 +47,13 @@ namespace dmr {
 
 namespace {
 
-constexpr int kR = 2;                                        // 16-feature tiles per consumer warp
-constexpr int kRowBlocks = 128 / (16 * kR);                  // consumer warps side by side over the features
-constexpr int kConsumerWarps = 2 * kRowBlocks;               // two k halves
-constexpr int kPublishWarp = kConsumerWarps + 1;            // one lane counts this CTA into shared feature groups
-constexpr int kStreamThreads = (kConsumerWarps + 2) * 32;  // + one producer warp + the publishing warp
+// Warp geometry.  8 consumer warps of 32 features each, except the 16-row kernel for bf16 weights: it has
+// its SM alone and no unpack work to amortise, and runs faster with 16 consumer warps of 16 features
+// (measured: +7 %; the 16-row kernels for packed codes lose 6 % that way and keep 8 warps).
+__host__ __device__ constexpr int r_tiles(int nt, int bits) { return (nt == 2 && bits == 16) ? 1 : 2; }  // 16-feature tiles per consumer warp
+__host__ __device__ constexpr int row_blocks(int nt, int bits) { return 128 / (16 * r_tiles(nt, bits)); }  // consumer warps side by side
+__host__ __device__ constexpr int consumer_warps(int nt, int bits) { return 2 * row_blocks(nt, bits); }    // two k halves
+__host__ __device__ constexpr int stream_threads(int nt, int bits) { return (consumer_warps(nt, bits) + 2) * 32; }  // + producer + publishing warp
 constexpr int kTileRows = 128;                              // features per step
 constexpr int kStepBytes = kTileRows * 128;                 // weight bytes per step (16 KB)
 constexpr int kMaxStages = 12;
@@ -246,8 +248,8 @@ struct StreamCfg {
     static constexpr int PARK_BYTES = 2 * SUM_FLOATS * 4;    // two parking buffers, used in turn
     static constexpr int SCRATCH = PART_BYTES > PARK_BYTES ? PART_BYTES : PARK_BYTES;
     static constexpr int SZ_OFF = D * STAGE + SCRATCH;
-    static constexpr int SZ_WARP = 2 * 16 * kR * GS * 4;  // per consumer warp: two slots of (scale, zero) entries
-    static constexpr int BAR_OFF = SZ_OFF + kConsumerWarps * SZ_WARP;
+    static constexpr int SZ_WARP = 2 * 16 * r_tiles(NT, BITS) * GS * 4;  // per consumer warp: two slots of (scale, zero) entries
+    static constexpr int BAR_OFF = SZ_OFF + consumer_warps(NT, BITS) * SZ_WARP;
     static constexpr size_t SMEM = (size_t)BAR_OFF + 512 + 1024 /*alignment slack*/;
 };
 
@@ -258,12 +260,13 @@ struct StreamCfg {
 // sums through distributed shared memory (no trip through the L2); without it, CTAs take contiguous
 // step ranges and shared feature groups are summed through global memory by the last to arrive.
 template <int BITS, int NT, int GS, bool CE, bool OUT_F32, bool CL>
-__global__ void __launch_bounds__(kStreamThreads, NT == 1 ? 2 : 1)
+__global__ void __launch_bounds__(stream_threads(NT, BITS), NT == 1 ? 2 : 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ CUtensorMap xmap,
                      const StreamArgs a) {
     using Cfg = StreamCfg<BITS, NT, GS>;
     using Geo = StepGeom<BITS>;
-    constexpr int D = Cfg::D, SLOTS = Cfg::SLOTS, R = kR;
+    constexpr int D = Cfg::D, SLOTS = Cfg::SLOTS, R = r_tiles(NT, BITS);
+    constexpr int kRowBlocks = row_blocks(NT, BITS), kConsumerWarps = consumer_warps(NT, BITS), kPublishWarp = kConsumerWarps + 1;
     constexpr int kClusterSize = cluster_size(NT);
     constexpr bool LOWBIT = BITS != 16;
     constexpr int WPS = 4 / GS;  // 32-bit code words per lane, feature and group part
@@ -509,7 +512,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
 #pragma unroll
         for (int sg = 0; sg < GS; ++sg) {
             const uint32_t v = (src[sg][0] << 16) | src[sg][1] | (BITS == 4 ? 0x4300u : 0u);
-            asm volatile("st.shared.u32 [%0], %1;" ::"r"(sz_base + (uint32_t)(((slot * GS + sg) * 16 * R + lane) * 4)), "r"(v) : "memory");
+            if (lane < 16 * R)
+                asm volatile("st.shared.u32 [%0], %1;" ::"r"(sz_base + (uint32_t)(((slot * GS + sg) * 16 * R + lane) * 4)), "r"(v) : "memory");
         }
         __syncwarp();
     };
@@ -949,7 +953,7 @@ dmr_status_t launch_stream_cl(const CUtensorMap &wmap, const CUtensorMap &xmap, 
     static int max_clusters_on[64] = {};
     const int dev = current_device();
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(kStreamThreads, 1, 1);
+    cfg.blockDim = dim3(stream_threads(NT, BITS), 1, 1);
     cfg.dynamicSmemBytes = Cfg::SMEM;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
