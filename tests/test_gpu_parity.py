@@ -334,6 +334,35 @@ def test_lowbit_linear_host_matches_device_call():
 
 # ---------------- full-size shapes, sampled outputs ----------------
 
+def test_decode_launch_chains_are_repeatable():
+    """Back-to-back launches on one stream and one workspace (programmatic dependent launch lets a kernel
+    start while its predecessor drains): every repetition must give the bits of the first one, and that
+    one must match the oracle.  Mixes layers that take the contiguous split (counters and partial sums
+    in the workspace) with layers that run in clusters, and 1-, 8- and 16-row batches."""
+    fmt = QFormat(4, 128)
+    cases = []
+    for (N, K, M) in [(3000, 11008, 1), (1024, 4096, 8), (3000, 11008, 16), (640, 2048, 16), (2200, 16384, 4)]:
+        W = inputs.weights(N, K, seed=21, index=N + M)
+        X = inputs.activations(M, K, seed=21, index=M + K)
+        q, ref = quantize_both(W, 4, 128)
+        Yref = oracle.lowbit_linear(X, *ref, bits=4, group=128)
+        cases.append((to_dev_bf16(X), q, Yref, torch.empty((M, N), dtype=torch.float32, device="cuda")))
+    ws = dmr.new_workspace(0, 16, 3000, 16384, fmt, "cuda")
+    first = []
+    for Xd, q, Yref, Y in cases:
+        dmr.dmr_lowbit_linear(Xd, q, OUT_F32, Y=Y, workspace=ws)
+        first.append(Y.clone())
+        assert rel_err(Y.cpu().numpy().astype(np.float64), Yref) <= TOL_ROUNDED
+    for rep in range(40):
+        outs = []
+        for Xd, q, Yref, Y in cases:
+            Yn = torch.empty_like(Y)
+            dmr.dmr_lowbit_linear(Xd, q, OUT_F32, Y=Yn, workspace=ws)
+            outs.append(Yn)
+        for Yn, Y0 in zip(outs, first):
+            assert torch.equal(Yn, Y0)
+
+
 @pytest.mark.parametrize("name,M", [("qkv", 1), ("o", 8), ("gate_up", 16), ("down", 16), ("gate_up", 4)])
 def test_7b_decode_shapes_sampled(name, M):
     N, K = inputs.LAYER_7B[name]
