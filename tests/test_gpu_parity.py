@@ -298,6 +298,24 @@ def test_routed_rows_move_between_chunks(M, N, K):
     routed_case(M, N, K, 4, 128, mask)
 
 
+@pytest.mark.parametrize("M", [12, 64])
+def test_routed_calls_in_a_row_are_repeatable(M):
+    """The two halves of a routed call run on two streams with scratch areas of their own; calls issued
+    back to back on one workspace must keep giving the bits of the first call."""
+    N, K = 1000, 4096
+    W = inputs.weights(N, K, seed=31, index=M)
+    X = inputs.activations(M, K, seed=31, index=M)
+    q, _ = quantize_both(W, 4, 128)
+    Xd, Wd = to_dev_bf16(X), to_dev_bf16(W)
+    masks = [torch.from_numpy(inputs.precision_mask(M, p, seed=7, index=i)).cuda() for i, p in enumerate((0.3, 0.7, 0.0, 1.0))]
+    ws = dmr.new_workspace(dmr.binding.OP_ROUTED, M, N, K, QFormat(4, 128), "cuda")
+    first = [dmr.dmr_routed_linear(Xd, m, Wd, q, OUT_F32, workspace=ws).clone() for m in masks]
+    for rep in range(15):
+        outs = [dmr.dmr_routed_linear(Xd, m, Wd, q, OUT_F32, workspace=ws) for m in masks]
+        for Yn, Y0 in zip(outs, first):
+            assert torch.equal(Yn, Y0)
+
+
 def test_routed_linear_prefill_sized_batch():
     # above 128 rows both the routed and the unrouted call take the persistent tensor-core kernel
     mask = inputs.precision_mask(300, 0.3, seed=15)
