@@ -96,8 +96,8 @@ dmr_status_t dmr_dequantize(const void *qweight, const void *scales, const void 
 
 /*
  * Low-precision linear layer (the W4A16 model's Linear, Sec. 5): Y = X . dequant(Wq)^T with fp32
- * accumulation.  Up to 32 rows run the bandwidth-bound decode kernel (in chunks of 16), larger M the
- * tensor-core kernels.
+ * accumulation.  Up to 32 rows run the bandwidth-bound decode kernel, larger M the tensor-core
+ * kernels.
  * M = 0 is a no-op.  workspace: dmr_workspace_bytes(DMR_OP_LOWBIT_LINEAR, ...) bytes.
  */
 dmr_status_t dmr_lowbit_linear(const void *X_bf16, int M, const void *qweight, const void *scales,

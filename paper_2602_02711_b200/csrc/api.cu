@@ -25,7 +25,7 @@ struct Scratch {
     void *prefill_scratch = nullptr;  // prepared fp16 activations and row scales of the prefill kernel
     float *partial = nullptr;
     void *stream_scratch = nullptr;  // counters + partial sums of the streaming decode kernel
-    uint16_t *xg_stream = nullptr;   // routed, decode path: 16 gathered activation rows
+    uint16_t *xg_stream = nullptr;   // routed, decode path: the gathered activation rows of one chunk
     // routed calls run their two halves on two streams: the high-precision half gets its own scratch
     float *partial_high = nullptr;
     void *stream_scratch_high = nullptr;
@@ -33,7 +33,9 @@ struct Scratch {
     size_t bytes = 0;
 };
 
-// Batches of up to this many rows stay on the streaming decode kernel (in chunks of 16 rows).  The
+constexpr int kStreamChunk = 32;  // rows one launch of the streaming decode kernel takes at most
+
+// Batches of up to this many rows stay on the streaming decode kernel (in chunks of 32 rows).  The
 // default is 32 (two chunks; measured faster than the tensor-core kernels up to there); the environment variable DMR_DECODE_MAX_M moves the crossover for measurements.
 int decode_max_m() {
     static int v = -1;
@@ -97,11 +99,11 @@ Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f
         off += round_up(stream_scratch_bytes(N), 256);
         if (op == DMR_OP_ROUTED_LINEAR) {
             s.xg_stream = reinterpret_cast<uint16_t *>(base + off);
-            off += round_up((size_t)16 * K * 2, 256);
+            off += round_up((size_t)kStreamChunk * K * 2, 256);
             s.stream_scratch_high = base + off;
             off += round_up(stream_scratch_bytes(N), 256);
             s.xg_stream_high = reinterpret_cast<uint16_t *>(base + off);
-            off += round_up((size_t)16 * K * 2, 256);
+            off += round_up((size_t)kStreamChunk * K * 2, 256);
         }
     }
     s.bytes = round_up(off, 256);
@@ -135,10 +137,10 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
         }
         return launch_gemm(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.partial, ws.status, st);
     }
-    if (!stream_supported(M < 16 ? M : 16, N, K, f.bits, g))
+    if (!stream_supported(M < kStreamChunk ? M : kStreamChunk, N, K, f.bits, g))
         return launch_simple_lowbit(X, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, st);
-    for (int m0 = 0; m0 < M; m0 += 16) {
-        const int mc = M - m0 < 16 ? M - m0 : 16;
+    for (int m0 = 0; m0 < M; m0 += kStreamChunk) {
+        const int mc = M - m0 < kStreamChunk ? M - m0 : kStreamChunk;
         RowSel s = sel;
         const uint16_t *Xc = X;
         void *Yc = Y;
@@ -173,9 +175,9 @@ dmr_status_t run_dense(const uint16_t *X, int M, RowSel sel, const uint16_t *W, 
         }
         return launch_gemm(Xin, M, sel, W, nullptr, nullptr, N, K, 0, K, Y, out, ws.partial, ws.status, st);
     }
-    if (!stream_supported(M < 16 ? M : 16, N, K, 16, K)) return launch_simple_dense(X, M, sel, W, N, K, Y, out, st);
-    for (int m0 = 0; m0 < M; m0 += 16) {
-        const int mc = M - m0 < 16 ? M - m0 : 16;
+    if (!stream_supported(M < kStreamChunk ? M : kStreamChunk, N, K, 16, K)) return launch_simple_dense(X, M, sel, W, N, K, Y, out, st);
+    for (int m0 = 0; m0 < M; m0 += kStreamChunk) {
+        const int mc = M - m0 < kStreamChunk ? M - m0 : kStreamChunk;
         RowSel s = sel;
         const uint16_t *Xc = X;
         void *Yc = Y;

@@ -70,7 +70,7 @@ constexpr int kCounterStride = 32;  // int32 words between counters
 size_t stream_scratch_bytes(int N);
 bool stream_supported(int M, int N, int K, int bits, int g);
 // `batch_rows` = rows of the whole call this launch is a chunk of (0 = M).  It alone decides between the
-// 8-row and the 16-row kernel, so that every row of a call goes through the same kernel (and the same
+// 8-, 16- and 32-row kernel, so that every row of a call goes through the same kernel (and the same
 // summation order) whichever chunk it falls into - a routed call moves rows between chunks.
 dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,
                            const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,

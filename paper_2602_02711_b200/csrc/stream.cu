@@ -1,4 +1,4 @@
-// Decode-time linear layers (M <= 16 rows): one persistent kernel that streams the weight matrix
+// Decode-time linear layers (up to 32 rows per launch): one persistent kernel that streams the weight matrix
 // exactly once at memory speed.  Decoding re-streams the model weights for every generated token
 // and is limited by memory bandwidth, which is where weight-only quantization pays (App.
 // "Evaluation protocol", discussion of output length; App. "Latency coefficients").
@@ -14,20 +14,20 @@
 //    with their next steps, and the sums of the groups a CTA was last for are formed at the end of the
 //    kernel by all consumer warps.
 //  - Small layers (up to 25 MB of codes), where that sum across CTAs is most of the run time:
-//    thread-block clusters of eight CTAs (four for the 16-row kernels).  A cluster owns whole feature
+//    thread-block clusters of eight CTAs (four for the 16- and 32-row kernels).  A cluster owns whole feature
 //    groups, rank r streams the r-th part of their k range, and at the end the cluster adds the sums
 //    of every output in rank order through distributed shared memory, each CTA taking its share of the
 //    outputs.
 // Either way there are no floating-point atomics, and the summation order of an output depends on
-// (N, K), the device and whether the call has up to 8 rows or more - never on the row's position in
-// the batch or on the other rows (all chunks of a call with more than 16 rows use the 16-row kernel).
+// (N, K), the device and whether the call has up to 8, up to 16 or more rows - never on the row's
+// position in the batch or on the other rows (all chunks of a call use the same kernel instance).
 //
 // Inside a CTA one producer lane keeps a ring of stages full by TMA (cp.async.bulk.tensor,
 // 128-byte swizzle): the weight box and the matching activation boxes, all completing on the
 // stage's mbarrier (a routed batch is gathered into consecutive rows beforehand).  Eight consumer
 // warps each own 32 features and one half of the step's k range; the product runs on the tensor
-// cores with the weights as the 16-row operand of mma.m16n8k16 and up to 8 (or 2 x 8) activation
-// rows as the 8-column operand.  4-bit codes are unpacked with one
+// cores with the weights as the 16-row operand of mma.m16n8k16 and 8 activation rows (one, two or
+// four such tiles per instance) as the 8-column operand.  4-bit codes are unpacked with one
 // LOP3 per two codes ((w >> 4p) & 0x000F000F | 0x43004300 = {128 + q_p, 128 + q_{p+4}} as two
 // bf16) and one packed subtract of (128 + zero): the tensor-core operand is the exact integer
 // q - zero.  Products are accumulated per quantization group in fp32 and the group's scale is
@@ -63,7 +63,7 @@ __host__ __device__ constexpr int cluster_size(int nt) { return nt == 1 ? 8 : 4;
 constexpr int kClusterMaxStepsDense = 2100;                // the same for bf16 weights (a 4096 x 4096 layer: 10.7 us instead of 13.9)
 constexpr int kClusterMaxSteps = 1600;                     // layers of up to this many steps (25 MB) run in cluster mode
 // Shared memory for the stage ring, KB: two 8-row CTAs share an SM, a 16-row CTA has it alone.
-__host__ __device__ constexpr int stage_budget_kb(int nt) { return nt == 1 ? 92 : 100; }
+__host__ __device__ constexpr int stage_budget_kb(int nt) { return nt == 1 ? 92 : (nt == 2 ? 100 : 136); }
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                                uint32_t a3, uint32_t b0, uint32_t b1) {
@@ -163,7 +163,7 @@ struct StreamArgs {
     int steps_per_group;      // ceil(K / STEP_K)
     int total_steps;          // feature groups * steps_per_group
     int part_groups;          // cluster mode: feature groups whose sums fit into a CTA's shared memory at once
-    int wide;                 // host side: 1 = the 16-row kernel (the call has more than 8 rows)
+    int tiles;                // host side: 8-row activation tiles of the kernel to launch (1, 2 or 4)
 };
 
 __device__ __forceinline__ long long range_begin(int c, int ctas, int total) {
@@ -244,7 +244,7 @@ struct StreamCfg {
     static constexpr int D = D_RAW > kMaxStages ? kMaxStages : D_RAW;
     static constexpr int SUM_FLOATS = SLOTS * kTileRows;     // the sums k half 1 parks for k half 0
     // cluster mode keeps the sums of several feature groups here until the cluster adds them up
-    static constexpr int PART_BYTES = NT == 1 ? (BITS == 16 ? 16 : 20) * 1024 : 64 * 1024;
+    static constexpr int PART_BYTES = NT == 1 ? (BITS == 16 ? 16 : 20) * 1024 : 64 * 1024;  // 4 to 40 groups at full row count
     static constexpr int PARK_BYTES = 2 * SUM_FLOATS * 4;    // two parking buffers, used in turn
     static constexpr int SCRATCH = PART_BYTES > PARK_BYTES ? PART_BYTES : PARK_BYTES;
     static constexpr int SZ_OFF = D * STAGE + SCRATCH;
@@ -253,7 +253,7 @@ struct StreamCfg {
     static constexpr size_t SMEM = (size_t)BAR_OFF + 512 + 1024 /*alignment slack*/;
 };
 
-// BITS: 4 / 8 = packed codes, 16 = bf16 weights.  NT: 8-row activation tiles (1 or 2).
+// BITS: 4 / 8 = packed codes, 16 = bf16 weights.  NT: 8-row activation tiles (1, 2 or 4).
 // GS: quantization groups per 128-code unit (2 only for 4-bit codes with 64-wide groups).
 // CE: every unit a warp consumes ends its quantization group (group size == unit size).
 // CL: the CTAs of a thread-block cluster split the k range of the same feature groups and add their
@@ -268,6 +268,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
     constexpr int D = Cfg::D, SLOTS = Cfg::SLOTS, R = r_tiles(NT, BITS);
     constexpr int kRowBlocks = row_blocks(NT, BITS), kConsumerWarps = consumer_warps(NT, BITS), kPublishWarp = kConsumerWarps + 1;
     constexpr int kClusterSize = cluster_size(NT);
+    constexpr int kPartSlots = NT == 4 ? 32 : 16;  // batch slots of a CTA's part of a shared feature group in global memory
     constexpr bool LOWBIT = BITS != 16;
     constexpr int WPS = 4 / GS;  // 32-bit code words per lane, feature and group part
     extern __shared__ uint8_t smem_dyn[];
@@ -777,7 +778,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
             if (kh == 0) {
                 // and writes the outputs (group owned alone) or this CTA's part of a shared group
                 const int which = beg > rg * SPG ? 0 : 1;
-                float *mine = a.partial + ((size_t)cta * 2 + which) * (16 * kTileRows);
+                float *mine = a.partial + ((size_t)cta * 2 + which) * (kPartSlots * kTileRows);
 #pragma unroll
                 for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -884,7 +885,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_cons
                 for (int u = 0; u < PF; ++u) {
                     const int cj = min(cj0 + u, c_last);
                     const int wj = range_begin(cj, ctas, a.total_steps) > s_first ? 0 : 1;
-                    p[u] = __ldcg(reinterpret_cast<const float4 *>(a.partial + ((size_t)cj * 2 + wj) * (16 * kTileRows)) + o4);
+                    p[u] = __ldcg(reinterpret_cast<const float4 *>(a.partial + ((size_t)cj * 2 + wj) * (kPartSlots * kTileRows)) + o4);
                 }
 #pragma unroll
                 for (int u = 0; u < PF; ++u)
@@ -1041,9 +1042,13 @@ dmr_status_t launch_stream_t(const CUtensorMap &wmap, const CUtensorMap &xmap, c
 template <int BITS, int GS, bool CE>
 dmr_status_t launch_stream_nt(const CUtensorMap &wmap, const CUtensorMap &xmap, const StreamArgs &a, int ctas,
                               dmr_out_t out, cudaStream_t st) {
-    if (!a.wide) {
+    if (a.tiles == 1) {
         if (out == DMR_OUT_F32) return launch_stream_t<BITS, 1, GS, CE, true>(wmap, xmap, a, ctas, st);
         return launch_stream_t<BITS, 1, GS, CE, false>(wmap, xmap, a, ctas, st);
+    }
+    if (a.tiles == 4) {
+        if (out == DMR_OUT_F32) return launch_stream_t<BITS, 4, GS, CE, true>(wmap, xmap, a, ctas, st);
+        return launch_stream_t<BITS, 4, GS, CE, false>(wmap, xmap, a, ctas, st);
     }
     if (out == DMR_OUT_F32) return launch_stream_t<BITS, 2, GS, CE, true>(wmap, xmap, a, ctas, st);
     return launch_stream_t<BITS, 2, GS, CE, false>(wmap, xmap, a, ctas, st);
@@ -1058,7 +1063,7 @@ size_t stream_scratch_bytes(int N) {
 
 bool stream_supported(int M, int N, int K, int bits /*16 = bf16 weights*/, int g) {
     (void)N;
-    if (M < 1 || M > 16) return false;
+    if (M < 1 || M > 32) return false;
     if (bits == 16) return K % 8 == 0;
     if (bits == 4) return g % 128 == 0 || g == 64;
     if (bits == 8) return g % 64 == 0;
@@ -1070,7 +1075,8 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
                            void *scratch, int32_t *status, cudaStream_t st, int batch_rows) {
     const int step_k = 1024 / bits;
     StreamArgs a;
-    a.wide = (batch_rows > M ? batch_rows : M) > 8 ? 1 : 0;
+    const int call_rows = batch_rows > M ? batch_rows : M;
+    a.tiles = call_rows <= 8 ? 1 : (call_rows <= 16 ? 2 : 4);
     a.idx = sel.idx;
     a.count = sel.count;
     a.scales = scales;
@@ -1093,7 +1099,8 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     if (total > 0x7FFFFFFF) return DMR_ERR_UNSUPPORTED;
     a.total_steps = (int)total;
     a.part_groups = 0;
-    int ctas = sm_count() * (a.wide ? 1 : 2);  // the 8-row kernels fit twice on an SM
+    int ctas = sm_count() * (a.tiles == 1 ? 2 : 1);  // the 8-row kernels fit twice on an SM
+    if (a.tiles == 4 && ctas > kMaxStreamCtas / 2) ctas = kMaxStreamCtas / 2;  // 32-slot parts are twice as large
     if (ctas > kMaxStreamCtas) ctas = kMaxStreamCtas;
     if (ctas > a.total_steps) ctas = a.total_steps;
     CUtensorMap wmap;
@@ -1104,7 +1111,7 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     // X holds M consecutive rows (for a routed call: the gathered rows); box = [8 or 16 slots][64 k]
     CUtensorMap xmap;
     if (!make_tensor_map_2d(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, (uint64_t)M, (uint64_t)K, (uint64_t)K * 2,
-                            a.wide ? 16 : 8, 64, TmaSwizzle::k128B))
+                            8 * a.tiles, 64, TmaSwizzle::k128B))
         return DMR_ERR_CUDA;
     if (bits == 16) return launch_stream_nt<16, 1, false>(wmap, xmap, a, ctas, out, st);
     if (bits == 8) {

@@ -139,6 +139,10 @@ def test_config1_lowbit_linear(M):
     (16, 328, 512, 8, 128),
     (1, 24, 128, 4, 128),      # smallest K the decode kernel takes
     (2, 40, 160, 4, 32),       # K not a multiple of 128: any-shape kernel
+    (24, 1000, 1024, 4, 128),  # 17 .. 32 rows: the 32-row instance of the decode kernel
+    (32, 520, 2048, 8, 0),
+    (17, 4096, 4096, 4, 64),   # ... in cluster mode (clusters of four)
+    (31, 22016, 512, 4, 128),  # ... with more feature groups per cluster than fit at once
     (40, 300, 512, 4, 128),    # M above the decode limit: tensor-core GEMM, ragged N and M
     (33, 136, 384, 8, 0),
     (64, 256, 4096, 4, 128),   # few tiles, long K: split-K with ordered reduction
@@ -190,7 +194,7 @@ def test_lowbit_linear_with_outlier_channels():
     run_lowbit_case(8, 512, 5120, 4, 64, seed=4, outlier=0.01)
 
 
-@pytest.mark.parametrize("M,N,K", [(1, 512, 512), (4, 512, 512), (16, 1000, 1024), (11, 72, 4096),
+@pytest.mark.parametrize("M,N,K", [(1, 512, 512), (4, 512, 512), (16, 1000, 1024), (11, 72, 4096), (27, 1000, 2048),
                                    (3, 40, 200), (40, 300, 512), (64, 256, 4096), (200, 264, 1024),
                                    (300, 520, 640), (1000, 130, 192)])
 def test_dense_linear(M, N, K):
