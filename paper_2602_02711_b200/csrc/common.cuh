@@ -60,7 +60,7 @@ dmr_status_t launch_dequantize(const uint32_t *qweight, const uint16_t *scales, 
                                int N, int K, int bits, int g, void *W_out, dmr_out_t out,
                                cudaStream_t st);
 
-// Streaming decode kernel (M <= 16): persistent, one CTA per SM, weights read once.  `bits` is 4 or 8
+// Streaming decode kernel (M <= 32 per launch): persistent, one or two CTAs per SM, weights read once.  `bits` is 4 or 8
 // for packed codes and 16 for bf16 weights.  `scratch` holds stream_scratch_bytes(N) bytes that are
 // zero before the first use (the kernel leaves its counters zeroed again).
 constexpr int kMaxStreamCtas = 512;
