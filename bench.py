@@ -523,10 +523,10 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
 
     if "crossover" in sections:
         # 32B-class gate and down linears, INT4 g=64 and INT8 per-channel, M = 1 .. 256, 1 % outlier channels x20:
-        # where the library's dispatch (streaming kernel up to 16 rows, tensor-core kernels above) stands.
+        # where the library's dispatch (streaming kernel up to 32 rows, tensor-core kernels above) stands.
         # The streaming family at larger M is timed by separate runs with DMR_DECODE_MAX_M=256.
         from paper_2602_02711_b200 import QFormat as QF
-        cx = {"dispatch": f"DMR_DECODE_MAX_M={os.environ.get('DMR_DECODE_MAX_M', '16')}"}
+        cx = {"dispatch": f"DMR_DECODE_MAX_M={os.environ.get('DMR_DECODE_MAX_M', '32')}"}
         for lname, (N, K) in inputs.LAYER_32B.items():
             for fname, f5 in (("int4_g64", QF(4, 64)), ("int8_pc", QF(8, 0))):
                 Ws = [randw(N, K, 61 + c) for c in range(2)]
