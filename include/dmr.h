@@ -96,8 +96,11 @@ dmr_status_t dmr_dequantize(const void *qweight, const void *scales, const void 
 
 /*
  * Low-precision linear layer (the W4A16 model's Linear, Sec. 5): Y = X . dequant(Wq)^T with fp32
- * accumulation.  Up to 32 rows run the bandwidth-bound decode kernel, larger M the tensor-core
- * kernels.
+ * accumulation.  Up to 32 rows run the bandwidth-bound decode kernels, larger M the tensor-core
+ * kernels.  The decode kernels start fetching qweight, scales and zeros before the preceding kernel
+ * of `stream` has finished (programmatic dependent launch): these three must be complete when the
+ * call is enqueued, or be written by kernels that do not release their dependents early (dmr_quantize
+ * and every ordinary kernel launch qualify).  X may be produced by the preceding kernel.
  * M = 0 is a no-op.  workspace: dmr_workspace_bytes(DMR_OP_LOWBIT_LINEAR, ...) bytes.
  */
 dmr_status_t dmr_lowbit_linear(const void *X_bf16, int M, const void *qweight, const void *scales,
@@ -156,7 +159,9 @@ dmr_status_t dmr_lowbit_linear_host(const void *X_host, int M, const void *qweig
  *   - Limits: 1 <= M <= 16, N <= dmr_noalloc_max_n() (65536), formats the decode kernel takes
  *     (4-bit with group 64 or a multiple of 128, 8-bit with a multiple of 64); anything else
  *     returns DMR_ERR_UNSUPPORTED and launches nothing.  X, qweight, scales, zeros and Y are the
- *     caller's device buffers exactly as for dmr_lowbit_linear; the result is identical to it.
+ *     caller's device buffers exactly as for dmr_lowbit_linear.  It always runs the shared-memory-ring
+ *     streaming kernel, so its result agrees with dmr_lowbit_linear's up to the order of the fp32 sums
+ *     (a few 1e-6 of the largest output), not bit for bit.
  *   - The first call on each device looks up the array's device address (no allocation); make
  *     that first call with the device current and before any stream capture begins.
  *   - The call allocates and frees nothing.  It clears the status word itself; all calls on one
@@ -192,6 +197,14 @@ dmr_status_t dmr_stepwise_kl(const void *logits_high, const void *logits_low, dm
 /* Reads the status word a previous call may have set in `workspace` (DMR_OK or DMR_ERR_TIMEOUT).
  * Synchronises `stream`. */
 dmr_status_t dmr_workspace_status(const void *workspace, void *stream);
+
+/*
+ * Writes a one-line description of the kernel family and launch shape that dmr_lowbit_linear
+ * (op = DMR_OP_LOWBIT_LINEAR) or dmr_dense_linear (DMR_OP_DENSE_LINEAR; f is ignored) would use for these sizes
+ * on the current device, e.g. "prefill bits=4 bn=256 tiles=3072 ctas=148".  Launches nothing.  Returns the length
+ * snprintf reports, or -1 for invalid arguments.  For tests and benchmarks that must know which kernel they ran.
+ */
+int dmr_describe_dispatch(dmr_op_t op, int M, int N, int K, dmr_qformat_t f, char *buf, size_t buf_bytes);
 
 const char *dmr_status_string(dmr_status_t s);
 int dmr_last_cuda_error(void);

@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
     L.dmr_lowbit_linear_noalloc.argtypes = [vp, i32, vp, vp, vp, i32, i32, QFormat, vp, i32, vp]
     L.dmr_workspace_status.restype = i32
     L.dmr_workspace_status.argtypes = [vp, vp]
+    L.dmr_describe_dispatch.restype = i32
+    L.dmr_describe_dispatch.argtypes = [i32, i32, i32, i32, QFormat, ctypes.c_char_p, sz]
     L.dmr_status_string.restype = ctypes.c_char_p
     L.dmr_status_string.argtypes = [i32]
     L.dmr_last_cuda_error.restype = i32
@@ -112,6 +114,21 @@ def _dev(t: torch.Tensor, dtype, name: str):
 
 def dmr_launch_count() -> int:
     return int(lib().dmr_launch_count())
+
+
+def dmr_describe_dispatch(op: int, M: int, N: int, K: int, fmt: QFormat = None) -> dict:
+    """Which kernel family and launch shape the library would use, as a dict such as
+    {"kernel": "prefill", "bits": 4, "bn": 256, "tiles": 3072, "ctas": 148}."""
+    buf = ctypes.create_string_buffer(256)
+    n = lib().dmr_describe_dispatch(op, M, N, K, fmt if fmt is not None else QFormat(4, 0), buf, 256)
+    if n < 0:
+        raise DmrError(1, "invalid arguments")
+    words = buf.value.decode().split()
+    out = {"kernel": words[0]}
+    for w in words[1:]:
+        k, v = w.split("=")
+        out[k] = int(v)
+    return out
 
 
 def dmr_workspace_bytes(op: int, M: int, N: int, K: int, fmt: QFormat) -> int:

@@ -1,6 +1,7 @@
 // C ABI of libdmr: argument validation, kernel-family choice and workspace carving.
 // Every entry point validates first and launches afterwards; nothing here synchronises the host
 // except dmr_workspace_status.
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
@@ -46,6 +47,19 @@ int decode_max_m() {
     }
     return v;
 }
+
+// The warp-ring decode kernel takes the 4-bit decode batches unless the environment says DMR_DECODE_KERNEL=stream
+// (the shared-memory ring kernel, kept for 8-bit codes, bf16 weights and for comparison).
+bool decode_w4_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("DMR_DECODE_KERNEL");
+        v = (e && strcmp(e, "stream") == 0) ? 0 : 1;
+    }
+    return v != 0;
+}
+
+constexpr int kDecodeChunk = 16;  // rows one launch of the 4-bit decode kernel takes at most
 
 bool use_gemm(int M, int N, int K, int bits, int g) { return M > decode_max_m() && gemm_supported(M, N, K, bits, g); }
 
@@ -136,6 +150,25 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
             Xin = ws.xg_low;
         }
         return launch_gemm(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.partial, ws.status, st);
+    }
+    if (f.bits == 4 && decode_w4_enabled() && decode_w4_supported(M < kDecodeChunk ? M : kDecodeChunk, N, K, g)) {
+        // chunks of up to 16 rows; the kernel gathers the rows of a routed call itself
+        for (int m0 = 0; m0 < M; m0 += kDecodeChunk) {
+            const int mc = M - m0 < kDecodeChunk ? M - m0 : kDecodeChunk;
+            RowSel s = sel;
+            const uint16_t *Xc = X;
+            void *Yc = Y;
+            if (sel.idx) {
+                s.idx = sel.idx + m0;
+                s.offset = sel.offset + m0;
+            } else {
+                Xc = X + (size_t)m0 * K;
+                Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
+            }
+            dmr_status_t r = launch_decode_w4(Xc, mc, s, qweight, scales, zeros, N, K, g, Yc, out, ws.status, st, M);
+            if (r != DMR_OK) return r;
+        }
+        return DMR_OK;
     }
     if (!stream_supported(M < kStreamChunk ? M : kStreamChunk, N, K, f.bits, g))
         return launch_simple_lowbit(X, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, st);
@@ -421,6 +454,36 @@ dmr_status_t dmr_workspace_status(const void *workspace, void *stream) {
         return DMR_ERR_CUDA;
     }
     return v == 0 ? DMR_OK : (dmr_status_t)v;
+}
+
+int dmr_describe_dispatch(dmr_op_t op, int M, int N, int K, dmr_qformat_t f, char *buf, size_t buf_bytes) {
+    if (!buf || buf_bytes == 0 || M < 1 || N < 1 || K < 1) return -1;
+    const bool dense = op == DMR_OP_DENSE_LINEAR;
+    if (op != DMR_OP_LOWBIT_LINEAR && op != DMR_OP_DENSE_LINEAR) return -1;
+    if (!dense && !format_ok(K, f)) return -1;
+    const int bits = dense ? 0 : f.bits, g = dense ? K : group_of(K, f);
+    if (use_gemm(M, N, K, bits, g)) {
+        if (!dense && prefill_supported(M, N, K, bits, g)) {
+            int bn, ctas;
+            long long tiles;
+            prefill_plan(M, N, &bn, &tiles, &ctas);
+            return snprintf(buf, buf_bytes, "prefill bits=%d bn=%d tiles=%lld ctas=%d", bits, bn, tiles, ctas);
+        }
+        const GemmPlan p = gemm_plan(M, N, K, bits);
+        return snprintf(buf, buf_bytes, "gemm bits=%d bn=%d splits=%d", bits, p.bn, p.splits);
+    }
+    if (!dense && bits == 4 && decode_w4_enabled() && decode_w4_supported(M < kDecodeChunk ? M : kDecodeChunk, N, K, g)) {
+        int nt, r, warps;
+        decode_w4_plan(M, g, &nt, &r, &warps);
+        return snprintf(buf, buf_bytes, "decode_w4 rows=%d tile=%d warps=%d chunks=%d", 8 * nt, 16 * r, warps, (M + kDecodeChunk - 1) / kDecodeChunk);
+    }
+    const int sbits = dense ? 16 : bits;
+    if (!stream_supported(M < kStreamChunk ? M : kStreamChunk, N, K, sbits, g)) return snprintf(buf, buf_bytes, "simple bits=%d", sbits);
+    int tiles, cluster;
+    long long steps;
+    stream_plan(M < kStreamChunk ? M : kStreamChunk, N, K, sbits, &tiles, &steps, &cluster);
+    return snprintf(buf, buf_bytes, "stream bits=%d rows=%d steps=%lld cluster=%d chunks=%d", sbits, 8 * tiles, steps, cluster,
+                    (M + kStreamChunk - 1) / kStreamChunk);
 }
 
 const char *dmr_status_string(dmr_status_t s) {

@@ -67,6 +67,8 @@ constexpr int kMaxStreamCtas = 512;
 // Feature-group counters sit one per 128-byte line: counts into different groups then never queue up
 // behind each other in the L2.
 constexpr int kCounterStride = 32;  // int32 words between counters
+// Scratch layout: per-CTA partial sums [kMaxStreamCtas][2][16 slots][128 features] fp32 first, the counters after them.
+constexpr size_t kStreamPartialBytes = (size_t)kMaxStreamCtas * 2 * 16 * 128 * sizeof(float);
 size_t stream_scratch_bytes(int N);
 bool stream_supported(int M, int N, int K, int bits, int g);
 // `batch_rows` = rows of the whole call this launch is a chunk of (0 = M).  It alone decides between the
@@ -75,6 +77,19 @@ bool stream_supported(int M, int N, int K, int bits, int g);
 dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,
                            const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
                            void *scratch, int32_t *status, cudaStream_t st, int batch_rows = 0);
+
+// Decode kernel for 4-bit codes (M <= 16 per launch): every CTA owns whole output features and streams their codes
+// through warp-private TMA rings; no scratch memory beyond the status word.  sel.idx / sel.count select and
+// count the rows of a routed call (the kernel gathers and scatters itself).  `batch_rows` as above.
+bool decode_w4_supported(int M, int N, int K, int g);
+dmr_status_t launch_decode_w4(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales,
+                              const uint8_t *zeros, int N, int K, int g, void *Y, dmr_out_t out, int32_t *status,
+                              cudaStream_t st, int batch_rows = 0);
+
+// What the launchers would choose for a call (for dmr_describe_dispatch).
+void decode_w4_plan(int M, int g, int *nt, int *r, int *warps);
+void stream_plan(int M, int N, int K, int bits, int *tiles, long long *steps, int *cluster);
+void prefill_plan(int M, int N, int *bn, long long *tiles, int *ctas);
 
 // Persistent prefill GEMM (M > 32, low-bit weights); sel.idx maps batch slots to rows of X and Y, sel.count
 // says how many slots are valid.

@@ -1,0 +1,608 @@
+// Decode-time 4-bit linear layer (up to 16 rows per launch): the weight matrix is read exactly once at memory
+// speed.  Decoding re-streams the model weights for every generated token and is limited by memory
+// bandwidth, which is where weight-only quantization pays (App. "Evaluation protocol", discussion of output
+// length; App. "Latency coefficients").
+//
+// Work decomposition.  The output features are cut into tiles of 16 R rows; CTA c of a grid of one CTA per SM
+// owns a contiguous range of tiles and, for each of them, the whole k range, so no sum ever crosses a CTA:
+// there is no scratch memory, no counter and no wait on another CTA in this kernel.  Inside the CTA all warps
+// work on the same tile and split its k range in boxes of 256 input features (box b goes to warp b % WARPS).
+// The partial sums of every output are added in warp order through shared memory - a fixed order that depends
+// on the instance and the layer's shape only, so a row's result never depends on the batch around it.
+//
+// Data movement.  Every warp has a ring of its own in shared memory that one of its lanes keeps full with TMA
+// boxes of [16 R rows x 128 bytes] of packed codes (two or four chunks; rows past N read as zero; 128-byte
+// swizzle); nobody else reads it, so the only synchronisation is the warp's own mbarrier per stage.  The boxes
+// are as large as the tile allows because every box costs the SM's copy engine a fixed time of its own
+// (measured: about 70 cycles, whatever its size).  A tile's scales and zero points are two contiguous blocks
+// of the tables; one thread copies them to shared memory two tiles ahead (bulk copies) when the layer's shape
+// allows it, otherwise they are read from global memory where they are needed.  Activations come through the
+// L1 with ordinary loads issued one chunk ahead.
+//
+// Inner loop.  Lane (g, t) (g = lane / 4, t = lane % 4) takes WPL consecutive code words of two rows of each
+// 16-row block and the 8 WPL activations they meet for batch rows g (and g + 8 in the 16-row instance).
+// ((w >> 4p) & 0x000F000F) | 0x43004300 is the bf16 pair {128 + q_p, 128 + q_{p+4}} - exact - and goes to the
+// tensor cores as it is (mma.m16n8k16, the weights as the 16-row operand), a byte permute pairs the
+// activations the same way, and one more MMA with an all-ones operand gives the sum of the chunk's activations
+// per batch row.  A chunk never crosses a quantization group, so per chunk
+//     sum_k x_k s (q_k - z) = s (sum_k x_k (128 + q_k) - (128 + z) sum_k x_k)
+// is formed in fp32 from the two accumulators: no weight is rounded, the zero point costs nothing per weight,
+// and the error against exact arithmetic is fp32 summation of terms about thirty times the result (a few
+// 1e-7 of the largest output, measured).
+//
+// Launch chains.  The kernel lets its successor start at once (programmatic dependent launch) and asks for
+// more than half of an SM's shared memory, so that an SM never holds two CTAs of these kernels: the
+// successor's CTA moves in when this kernel's CTA on that SM has finished, asks for its share of the weights
+// to be brought into the L2 (bulk prefetches consume no value), fills its rings and only then waits for its
+// predecessor.  (With two CTAs per SM the successor's CTAs land wherever a slot happens to be free - two on
+// some SMs, none on others - and the kernel runs at the pace of the doubly loaded SMs; measured with in-kernel
+// time stamps.)  Weights, scales and zero points are read before the wait: they must not be produced by a
+// kernel that releases its dependents early (the library's own kernels that write weights never do).
+#include <cuda_bf16.h>
+
+#include <cstdlib>
+
+#include "sm100.cuh"
+
+namespace dmr {
+
+namespace {
+
+constexpr int kPrefetchPiece = 4096;              // bytes per bulk prefetch instruction
+constexpr long long kPrefetchAhead = 192 * 1024;  // bytes of weights a CTA keeps requested ahead of its loads
+
+struct DecodeArgs {
+    const uint16_t *X;        // [*][K] bf16
+    const int32_t *idx;       // routed: row of X / Y for batch slot s (nullptr = identity)
+    const int32_t *count;     // routed: valid slots in the whole list (nullptr = M)
+    const uint32_t *qweight;  // [N][K / 8]
+    const uint16_t *scales;   // [N][G] bf16
+    const uint8_t *zeros;     // [N][G]
+    void *Y;                  // [*][N]
+    int32_t *status;          // set to DMR_ERR_TIMEOUT if a bounded wait runs out
+    int M, coff, N, K, G;
+    int g_shift;              // log2(group size) when it is a power of two, else -1
+    int g_size;
+    int tiles;                // ceil(N / tile rows)
+    int nchunks;              // K / chunk size
+    int pf_tiles;             // tiles whose weights are requested ahead
+    int sz_stage;             // 1: a tile's scales and zero points are copied to shared memory ahead of time
+    int sz_vec;               // 1: the entries of a box's groups are consecutive, aligned and read with one load each
+    int sz_zoff, sz_stride;   // shared-memory offset of a tile's zero points; bytes between the tile buffers
+};
+
+__device__ __forceinline__ uint4 ldg_v4(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+// Asks the memory system to bring [p, p + bytes) into the L2; nothing is written anywhere else and
+// nothing waits for it.  p and bytes are multiples of 16.
+__device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void prefetch_l2_line(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+// Copies `bytes` (a multiple of 16, both addresses 16-byte aligned) from global to shared memory; completes on `bar`.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
+                 "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+constexpr size_t kMinSmem = 116 * 1024;  // more than half of the 228 KB of an SM
+constexpr int kSzBuffers = 3;  // tiles whose scales and zero points are in shared memory at a time
+
+template <int NT, int R, int WPL, int WARPS, int D>
+struct DecodeCfg {
+    static constexpr int THREADS = WARPS * 32;
+    static constexpr int TILE = 16 * R;
+    static constexpr int CHUNK_K = 32 * WPL;
+    static constexpr int CHUNK_BYTES = CHUNK_K / 2;
+    static constexpr int BOX_BYTES = 128;                     // bytes of a row in one TMA box (the 128-byte swizzle span)
+    static constexpr int CPB = BOX_BYTES / CHUNK_BYTES;       // chunks per box
+    static constexpr int STAGE_BYTES = TILE * BOX_BYTES;
+    static constexpr int NACC = R * NT * 4;
+    static constexpr int RING_BYTES = WARPS * D * STAGE_BYTES;
+    static constexpr int RED_BUFS = WARPS * NACC * 32 * 4 * 2 <= 32 * 1024 ? 2 : 1;  // one buffer costs a second barrier per tile
+    static constexpr int RED_BYTES = RED_BUFS * WARPS * NACC * 32 * 4;
+    static constexpr int BAR_OFF = RING_BYTES + RED_BYTES;     // WARPS * D ring barriers, then kSzBuffers table barriers
+    static constexpr int SZ_OFF = BAR_OFF + ((WARPS * D + kSzBuffers) * 8 + 15) / 16 * 16;
+    static constexpr size_t SMEM = (size_t)SZ_OFF + 1024 /*alignment slack*/;  // plus kSzBuffers * sz_stride when staging
+};
+
+// NT: 8-row activation blocks (1 or 2).  R: 16-row weight blocks per tile.  WPL: code words per lane and
+// row in one chunk (4: chunks of 128 input features, for groups that are multiples of 128; 2: chunks of
+// 64, for groups of 64).  WARPS: warps per CTA.  D: stages of a warp's ring.
+template <int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
+__global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_constant__ CUtensorMap wmap, const DecodeArgs a) {
+    using Cfg = DecodeCfg<NT, R, WPL, WARPS, D>;
+    constexpr int TILE = Cfg::TILE, CHUNK_K = Cfg::CHUNK_K, NACC = Cfg::NACC, THREADS = Cfg::THREADS, CPB = Cfg::CPB;
+    extern __shared__ uint8_t smem_dyn[];
+    const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    float *red = reinterpret_cast<float *>(smem_dyn + (base - smem_u32(smem_dyn)) + Cfg::RING_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    const int pg = (g >> 1) | ((g & 1) << 2);  // box row of fragment row g: 0, 4, 1, 5, ... (bank-conflict-free under the swizzle)
+    const int t0 = (int)(((long long)blockIdx.x * a.tiles) / gridDim.x);
+    const int t1 = (int)(((long long)(blockIdx.x + 1) * a.tiles) / gridDim.x);
+    const size_t row_bytes = (size_t)a.K >> 1;
+    const uint32_t ring = base + (uint32_t)warp * (D * Cfg::STAGE_BYTES);
+    const uint32_t bars = base + Cfg::BAR_OFF + (uint32_t)warp * (D * 8);
+    const uint32_t szbars = base + Cfg::BAR_OFF + WARPS * D * 8;
+    const uint32_t szbuf = base + Cfg::SZ_OFF;
+    const int nboxes = (a.nchunks + CPB - 1) / CPB;
+
+    if (lane == 0) {
+#pragma unroll
+        for (int d = 0; d < D; ++d) mbar_init(bars + 8 * d, 1);
+        if (warp == 0) {
+#pragma unroll
+            for (int d = 0; d < kSzBuffers; ++d) mbar_init(szbars + 8 * d, 1);
+            prefetch_tensor_map(&wmap);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+
+    // ---- requests for this CTA's weights, scales and zero points (no value is looked at) ----
+    auto prefetch_tiles = [&](int ta, int tb) {  // tiles [ta, tb)
+        const long long r0 = (long long)ta * TILE, r1 = min((long long)tb * TILE, (long long)a.N);
+        if (r1 <= r0) return;
+        const char *wb = reinterpret_cast<const char *>(a.qweight) + r0 * row_bytes;
+        const long long wbytes = (r1 - r0) * (long long)row_bytes;
+        for (long long o = (long long)threadIdx.x * kPrefetchPiece; o < wbytes; o += (long long)THREADS * kPrefetchPiece)
+            prefetch_l2_bulk(wb + o, (uint32_t)min((long long)kPrefetchPiece, wbytes - o));
+        const char *sb = reinterpret_cast<const char *>(a.scales) + r0 * a.G * 2;
+        const long long sbytes = (r1 - r0) * a.G * 2;
+        for (long long o = (long long)threadIdx.x * 128; o < sbytes; o += (long long)THREADS * 128) prefetch_l2_line(sb + o);
+        const char *zb = reinterpret_cast<const char *>(a.zeros) + r0 * a.G;
+        const long long zbytes = (r1 - r0) * a.G;
+        for (long long o = (long long)threadIdx.x * 128; o < zbytes; o += (long long)THREADS * 128) prefetch_l2_line(zb + o);
+    };
+    if (t1 > t0) prefetch_tiles(t0, min(t1, t0 + a.pf_tiles));
+
+    // ---- a tile's scales and zero points into shared memory (two contiguous blocks of the tables) ----
+    int sz_issued = 0;
+    auto issue_sz = [&](int tile) {  // by thread 0; tiles in the order this CTA takes them
+        if (!a.sz_stage || tile >= t1) return;
+        const int d = sz_issued % kSzBuffers;
+        const uint32_t n_entries = (uint32_t)(TILE * a.G);  // staging is only chosen when every tile is whole
+        mbar_expect_tx(szbars + 8 * d, n_entries * 3);
+        bulk_copy_g2s(szbuf + d * a.sz_stride, a.scales + (size_t)tile * n_entries, n_entries * 2, szbars + 8 * d);
+        bulk_copy_g2s(szbuf + d * a.sz_stride + a.sz_zoff, a.zeros + (size_t)tile * n_entries, n_entries, szbars + 8 * d);
+        ++sz_issued;
+    };
+    if (threadIdx.x == 0) {
+        issue_sz(t0);
+        issue_sz(t0 + 1);
+    }
+
+    // ---- this warp's list of steps: tiles t0, t0 + 1, ...; boxes warp, warp + WARPS, ... of each ----
+    const bool has_boxes = warp < nboxes;
+    bool ok = true;  // false once a bounded wait ran out: the warp stops copying, waiting and storing but still meets every barrier
+    int i_tile = t0, i_box = warp, issued = 0;  // the next box to request
+    auto issue = [&]() {
+        if (!has_boxes || i_tile >= t1 || !ok) return;
+        if (lane == 0) {
+            const int d = issued % D;
+            mbar_expect_tx(bars + 8 * d, Cfg::STAGE_BYTES);
+            tma_load_2d(ring + d * Cfg::STAGE_BYTES, &wmap, bars + 8 * d, i_box * Cfg::BOX_BYTES, i_tile * TILE);
+        }
+        ++issued;
+        i_box += WARPS;
+        if (i_box >= nboxes) {
+            i_box = warp;
+            ++i_tile;
+        }
+    };
+#pragma unroll
+    for (int d = 0; d < D; ++d) issue();
+
+    pdl_wait();
+    const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
+    if (rows <= 0 || t1 <= t0) {
+        // nothing to do (a routed call without rows of this kind): let the copies already under way land first
+        for (int d = 0; d < D && d < issued; ++d) mbar_wait(bars + 8 * d, 0u, a.status);
+        if (threadIdx.x == 0)
+            for (int d = 0; d < sz_issued; ++d) mbar_wait(szbars + 8 * d, 0u, a.status);
+        return;
+    }
+
+    // this lane's activation rows (batch slot nt * 8 + g; slots past the batch read the first row again: their
+    // columns of the products are never stored)
+    const uint16_t *xrow[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int slot = nt * 8 + g < rows ? nt * 8 + g : 0;
+        xrow[nt] = a.X + (size_t)(a.idx ? a.idx[slot] : slot) * a.K + t * (8 * WPL);
+    }
+    uint32_t x[NT][WPL][4];  // 8 activations per code word of the chunk to come
+    auto load_x = [&](int chunk) {
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int j = 0; j < WPL; ++j) {
+                const uint4 v = ldg_v4(xrow[nt] + chunk * CHUNK_K + 8 * j);
+                x[nt][j][0] = v.x;
+                x[nt][j][1] = v.y;
+                x[nt][j][2] = v.z;
+                x[nt][j][3] = v.w;
+            }
+    };
+    if (has_boxes) load_x(warp * CPB);
+
+    float acc[R][NT][4];
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[r][nt][c] = 0.f;
+
+    int consumed = 0;
+    constexpr uint32_t kOnes = 0x3F803F80u;  // bf16 1.0 twice
+    for (int tile = t0, tl = 0; tile < t1; ++tile, ++tl) {
+        // where the lane's rows' scales and zero points are: element offsets into the tables (global or the tile's copy)
+        uint32_t szo[R][2];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int n = min(tile * TILE + pg + r * 16 + h * 8, a.N - 1);
+                szo[r][h] = (uint32_t)(a.sz_stage ? n - tile * TILE : n) * (uint32_t)a.G;
+            }
+        const uint32_t sbase = szbuf + (uint32_t)(tl % kSzBuffers) * a.sz_stride, zbase = sbase + a.sz_zoff;
+        if (a.sz_stage && ok) ok = mbar_wait(szbars + 8 * (tl % kSzBuffers), (uint32_t)((tl / kSzBuffers) & 1), a.status);
+        for (int box = warp; box < nboxes; box += WARPS) {
+            const int d = consumed % D;
+            if (ok) ok = mbar_wait(bars + 8 * d, (uint32_t)((consumed / D) & 1), a.status);
+            ++consumed;
+            const uint32_t stage = ring + d * Cfg::STAGE_BYTES;
+            const int nsub = min(CPB, a.nchunks - box * CPB);
+            const int grp0 = a.g_shift >= 0 ? ((box * CPB * CHUNK_K) >> a.g_shift) : ((box * CPB * CHUNK_K) / a.g_size);
+            // scales and zero points of the box's groups when they sit side by side in the tile's copy
+            uint32_t scv[R][2][CPB / 2], zpv[R][2];
+            if (a.sz_vec) {
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t o = szo[r][h] + (uint32_t)grp0;
+                        if constexpr (CPB == 2) {
+                            scv[r][h][0] = lds_u32(sbase + 2 * o);
+                            zpv[r][h] = lds_u16(zbase + o);
+                        } else {
+                            const uint2 v = lds_v2(sbase + 2 * o);
+                            scv[r][h][0] = v.x;
+                            scv[r][h][CPB / 2 - 1] = v.y;
+                            zpv[r][h] = lds_u32(zbase + o);
+                        }
+                    }
+            }
+#pragma unroll
+            for (int sub = 0; sub < CPB; ++sub) {
+                if (sub >= nsub) break;
+                const int chunk = box * CPB + sub;
+                // scale (as fp32 bits) and zero point of this chunk's group for the lane's rows
+                uint32_t sc[R][2], zp[R][2];
+                if (a.sz_vec) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t pair = scv[r][h][sub / 2];
+                            sc[r][h] = (sub & 1) ? (pair & 0xFFFF0000u) : (pair << 16);
+                            zp[r][h] = (zpv[r][h] >> (8 * sub)) & 0xFFu;
+                        }
+                } else {
+                    const int k0 = chunk * CHUNK_K;
+                    const uint32_t grp = (uint32_t)(a.g_shift >= 0 ? (k0 >> a.g_shift) : (k0 / a.g_size));
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (a.sz_stage) {
+                                sc[r][h] = lds_u16(sbase + 2 * (szo[r][h] + grp)) << 16;
+                                zp[r][h] = lds_u8(zbase + szo[r][h] + grp);
+                            } else {
+                                sc[r][h] = (uint32_t)__ldg(a.scales + szo[r][h] + grp) << 16;
+                                zp[r][h] = __ldg(a.zeros + szo[r][h] + grp);
+                            }
+                        }
+                }
+                uint32_t w[R][2][WPL];
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t rowaddr = stage + (uint32_t)((r * 16 + h * 8 + pg) * Cfg::BOX_BYTES);
+                        if constexpr (WPL == 4) {
+                            const uint4 v = lds_v4(rowaddr + (uint32_t)(((sub * 4 + t) ^ pg) << 4));
+                            w[r][h][0] = v.x;
+                            w[r][h][1] = v.y;
+                            w[r][h][2 % WPL] = v.z;
+                            w[r][h][3 % WPL] = v.w;
+                        } else {
+                            const uint2 v = lds_v2(rowaddr + (uint32_t)((((sub * 2 + (t >> 1)) ^ pg) << 4) + (t & 1) * 8));
+                            w[r][h][0] = v.x;
+                            w[r][h][1] = v.y;
+                        }
+                    }
+                float gs[R][NT][4], sx[NT][4];
+#pragma unroll
+                for (int j = 0; j < WPL; ++j) {
+                    // activations paired like the codes: (x0, x4), (x1, x5) and (x2, x6), (x3, x7)
+                    uint32_t b[NT][4];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        b[nt][0] = prmt(x[nt][j][0], x[nt][j][2], 0x5410);
+                        b[nt][1] = prmt(x[nt][j][0], x[nt][j][2], 0x7632);
+                        b[nt][2] = prmt(x[nt][j][1], x[nt][j][3], 0x5410);
+                        b[nt][3] = prmt(x[nt][j][1], x[nt][j][3], 0x7632);
+                        if (j == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                        else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                        mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][2], b[nt][3]);
+                    }
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        uint32_t av[2][4];  // [pair of MMAs][a0..a3]: 128 + code, exact in bf16
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t u = w[r][h][j];
+                            av[0][h] = lop3_and_or(u, 0x000F000Fu, 0x43004300u);            // codes 0, 4
+                            av[0][2 + h] = lop3_and_or(u >> 4, 0x000F000Fu, 0x43004300u);   // codes 1, 5
+                            av[1][h] = lop3_and_or(u >> 8, 0x000F000Fu, 0x43004300u);       // codes 2, 6
+                            av[1][2 + h] = lop3_and_or(u >> 12, 0x000F000Fu, 0x43004300u);  // codes 3, 7
+                        }
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            if (j == 0) mma_bf16_16816_zero(gs[r][nt], av[0][0], av[0][1], av[0][2], av[0][3], b[nt][0], b[nt][1]);
+                            else mma_bf16_16816(gs[r][nt], av[0][0], av[0][1], av[0][2], av[0][3], b[nt][0], b[nt][1]);
+                            mma_bf16_16816(gs[r][nt], av[1][0], av[1][1], av[1][2], av[1][3], b[nt][2], b[nt][3]);
+                        }
+                    }
+                    if (j == 0 && sub == nsub - 1) {
+                        // one word of every shared-memory load of the box's last chunk has been used, so the stage
+                        // is in registers: request the box D ahead into it
+                        __syncwarp();
+                        issue();
+                    }
+                }
+                // the next chunk's activations
+                {
+                    int nc = chunk + 1;
+                    bool more = true;
+                    if (sub == nsub - 1) {
+                        if (box + WARPS < nboxes) nc = (box + WARPS) * CPB;
+                        else {
+                            nc = warp * CPB;
+                            more = tile + 1 < t1;
+                        }
+                    }
+                    if (more) load_x(nc);
+                }
+                // the chunk lies inside one quantization group: s (sum x (128 + q) - (128 + z) sum x)
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float s0 = __uint_as_float(sc[r][0]), s1 = __uint_as_float(sc[r][1]);
+                    const float z0 = __uint_as_float((zp[r][0] | 0x4300u) << 16), z1 = __uint_as_float((zp[r][1] | 0x4300u) << 16);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        acc[r][nt][0] = fmaf(s0, fmaf(-z0, sx[nt][0], gs[r][nt][0]), acc[r][nt][0]);
+                        acc[r][nt][1] = fmaf(s0, fmaf(-z0, sx[nt][1], gs[r][nt][1]), acc[r][nt][1]);
+                        acc[r][nt][2] = fmaf(s1, fmaf(-z1, sx[nt][2], gs[r][nt][2]), acc[r][nt][2]);
+                        acc[r][nt][3] = fmaf(s1, fmaf(-z1, sx[nt][3], gs[r][nt][3]), acc[r][nt][3]);
+                    }
+                }
+            }
+        }
+        // ---- end of a tile: add the warps' sums in warp order and write the outputs ----
+        if (tile + a.pf_tiles < t1) prefetch_tiles(tile + a.pf_tiles, tile + a.pf_tiles + 1);
+        float *rbuf = red + (size_t)(Cfg::RED_BUFS == 2 ? (tl & 1) : 0) * WARPS * (NACC * 32);
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    rbuf[(warp * NACC + (r * NT + nt) * 4 + c) * 32 + lane] = acc[r][nt][c];
+                    acc[r][nt][c] = 0.f;
+                }
+        __syncthreads();
+        // every warp is past this tile's table: its buffer takes the tile kSzBuffers - 1 further on
+        if (threadIdx.x == 0 && ok) issue_sz(tile + kSzBuffers - 1);
+        for (int o = threadIdx.x; o < NACC * 32; o += THREADS) {
+            const int e = o >> 5, l = o & 31;
+            float v = rbuf[e * 32 + l];
+#pragma unroll
+            for (int w2 = 1; w2 < WARPS; ++w2) v += rbuf[(w2 * NACC + e) * 32 + l];
+            const int c = e & 3, nt = (e >> 2) % NT, r = (e >> 2) / NT;
+            const int slot = nt * 8 + 2 * (l & 3) + (c & 1);
+            const int lg = l >> 2;
+            const int n = tile * TILE + r * 16 + ((lg >> 1) | ((lg & 1) << 2)) + 8 * (c >> 1);
+            if (ok && slot < rows && n < a.N) {
+                const int row = a.idx ? a.idx[slot] : slot;
+                if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
+                else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
+            }
+        }
+        if (Cfg::RED_BUFS == 1) __syncthreads();  // the sums are read before the next tile's overwrite them
+    }
+}
+
+int device_sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) cached[dev] = n;
+        else cached[dev] = 148;
+    }
+    return cached[dev];
+}
+
+bool decode_pdl_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("DMR_PDL");
+        v = (e && e[0] == '0') ? 0 : 1;
+    }
+    return v != 0;
+}
+
+template <int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
+dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
+    using Cfg = DecodeCfg<NT, R, WPL, WARPS, D>;
+    constexpr int TILE = Cfg::TILE;
+    // shared memory left for the copies of the scale / zero-point tables (227 KB per CTA at most)
+    constexpr size_t kSzBudget = 227 * 1024 - Cfg::SMEM < 36 * 1024 ? 227 * 1024 - Cfg::SMEM : 36 * 1024;
+    static_assert(Cfg::SMEM <= 227 * 1024, "ring and reduction buffers exceed an SM's shared memory");
+    auto kernel = decode_w4_kernel<NT, R, WPL, WARPS, D, OUT_F32>;
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    if (!configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(Cfg::SMEM + kSzBudget < kMinSmem ? kMinSmem : Cfg::SMEM + kSzBudget));
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            return DMR_ERR_CUDA;
+        }
+        configured[dev] = true;
+    }
+    a.tiles = (a.N + TILE - 1) / TILE;
+    a.nchunks = a.K / Cfg::CHUNK_K;
+    int ctas = device_sm_count();
+    if (ctas > a.tiles) ctas = a.tiles;
+    const long long tile_bytes = (long long)TILE * (a.K / 2);
+    a.pf_tiles = (int)((kPrefetchAhead + tile_bytes - 1) / tile_bytes);
+    if (a.pf_tiles < 2) a.pf_tiles = 2;
+    // A tile's scales and zero points are two contiguous blocks of the tables: they are copied to shared memory ahead
+    // of time when every tile is whole, the blocks are 16-byte aligned and three tiles' worth stay small.
+    const size_t tile_entries = (size_t)TILE * a.G;
+    a.sz_zoff = (int)((tile_entries * 2 + 15) / 16 * 16);
+    a.sz_stride = a.sz_zoff + (int)((tile_entries + 15) / 16 * 16);
+    a.sz_stage = (a.N % TILE == 0 && tile_entries % 16 == 0 && ((uintptr_t)a.scales % 16) == 0 && ((uintptr_t)a.zeros % 16) == 0 &&
+                  (size_t)kSzBuffers * a.sz_stride <= kSzBudget) ? 1 : 0;
+    // a box covers CPB consecutive groups and every row's entries start at a multiple of CPB
+    a.sz_vec = (a.sz_stage && a.g_size == Cfg::CHUNK_K && a.G % Cfg::CPB == 0) ? 1 : 0;
+    const size_t smem = Cfg::SMEM + (a.sz_stage ? (size_t)kSzBuffers * a.sz_stride : 0);
+    CUtensorMap wmap;
+    const uint64_t rb = (uint64_t)a.K / 2;
+    if (!make_tensor_map_2d(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.qweight, (uint64_t)a.N, rb, rb, TILE, Cfg::BOX_BYTES,
+                            TmaSwizzle::k128B))
+        return DMR_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas, 1, 1);
+    cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
+    // more than half of an SM's shared memory: two CTAs of these kernels never share an SM (see above)
+    cfg.dynamicSmemBytes = smem < kMinSmem ? kMinSmem : smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    int n_attr = 0;
+    if (decode_pdl_enabled()) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = (unsigned)n_attr;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, wmap, a);
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        (void)cudaGetLastError();
+        return DMR_ERR_CUDA;
+    }
+    return check_launch();
+}
+
+}  // namespace
+
+bool decode_w4_supported(int M, int N, int K, int g) {
+    (void)N;
+    if (M < 1 || M > 16) return false;
+    if (g == 64) return K % 64 == 0;
+    return g % 128 == 0 && K % 128 == 0;
+}
+
+// Instances as <NT, R, WPL, WARPS, D>.
+#ifndef DMR_DECODE_CFG8
+#define DMR_DECODE_CFG8 1, 2, 4, 16, 2
+#endif
+#ifndef DMR_DECODE_CFG8_G64
+#define DMR_DECODE_CFG8_G64 1, 2, 2, 16, 2
+#endif
+#ifndef DMR_DECODE_CFG16
+#define DMR_DECODE_CFG16 2, 2, 4, 8, 2
+#endif
+#ifndef DMR_DECODE_CFG16_G64
+#define DMR_DECODE_CFG16_G64 2, 2, 2, 8, 2
+#endif
+
+void decode_w4_plan(int M, int g, int *nt, int *r, int *warps) {
+    const int cfg8[5] = {DMR_DECODE_CFG8}, cfg8g[5] = {DMR_DECODE_CFG8_G64}, cfg16[5] = {DMR_DECODE_CFG16}, cfg16g[5] = {DMR_DECODE_CFG16_G64};
+    const int *c = M <= 8 ? (g == 64 ? cfg8g : cfg8) : (g == 64 ? cfg16g : cfg16);
+    *nt = c[0];
+    *r = c[1];
+    *warps = c[3];
+}
+
+dmr_status_t launch_decode_w4(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales,
+                              const uint8_t *zeros, int N, int K, int g, void *Y, dmr_out_t out, int32_t *status,
+                              cudaStream_t st, int batch_rows) {
+    DecodeArgs a = {};
+    a.X = X;
+    a.idx = sel.idx;
+    a.count = sel.count;
+    a.coff = sel.offset;
+    a.qweight = qweight;
+    a.scales = scales;
+    a.zeros = zeros;
+    a.Y = Y;
+    a.status = status;
+    a.M = M;
+    a.N = N;
+    a.K = K;
+    a.G = K / g;
+    a.g_size = g;
+    a.g_shift = -1;
+    for (int sh = 0; sh < 31; ++sh)
+        if ((1 << sh) == g) a.g_shift = sh;
+    const int call_rows = batch_rows > M ? batch_rows : M;
+    const bool f32 = out == DMR_OUT_F32;
+    if (call_rows <= 8) {
+        if (g == 64) return f32 ? launch_decode_t<DMR_DECODE_CFG8_G64, true>(a, st) : launch_decode_t<DMR_DECODE_CFG8_G64, false>(a, st);
+        return f32 ? launch_decode_t<DMR_DECODE_CFG8, true>(a, st) : launch_decode_t<DMR_DECODE_CFG8, false>(a, st);
+    }
+    if (g == 64) return f32 ? launch_decode_t<DMR_DECODE_CFG16_G64, true>(a, st) : launch_decode_t<DMR_DECODE_CFG16_G64, false>(a, st);
+    return f32 ? launch_decode_t<DMR_DECODE_CFG16, true>(a, st) : launch_decode_t<DMR_DECODE_CFG16, false>(a, st);
+}
+
+}  // namespace dmr

@@ -17,8 +17,7 @@ namespace {
 constexpr int kNoallocMaxN = 65536;
 constexpr size_t kNoallocStatusBytes = 256;
 constexpr size_t kNoallocScratchBytes =
-    kNoallocStatusBytes + (size_t)(kNoallocMaxN / 128) * kCounterStride * sizeof(int32_t) +
-    (size_t)kMaxStreamCtas * 2 * 16 * 128 * sizeof(float);
+    kNoallocStatusBytes + kStreamPartialBytes + (size_t)(kNoallocMaxN / 128) * kCounterStride * sizeof(int32_t);
 
 // In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocScratchBytes];

@@ -62,31 +62,6 @@ struct PrefillArgs {
     int n_tiles, m_tiles;
 };
 
-__device__ __forceinline__ uint32_t p_lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
-    uint32_t r;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));
-    return r;
-}
-__device__ __forceinline__ uint32_t p_prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t r;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-    return r;
-}
-__device__ __forceinline__ uint32_t p_sub_f16x2(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
-__device__ __forceinline__ uint32_t p_mul_f16x2(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
-__device__ __forceinline__ uint32_t p_pack_f16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 
 // Activation preparation: Xh[slot][k] = fp16(X[row(slot)][k] * 2^-e), xscale[slot] = 2^e, with e chosen
 // per row so that the row's largest magnitude lands in [2^13, 2^14).  Slots past the valid count
@@ -310,12 +285,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {  // word c = codes 8c .. 8c+7 = 16-byte chunk c of the row
                         const uint32_t w8 = w[c] >> 8;
-                        const uint32_t d04 = p_mul_f16x2(p_sub_f16x2(p_lop3_and_or(w[c], 0x000F000Fu, 0x64006400u), zoff), s2);
-                        const uint32_t d15 = p_mul_f16x2(p_sub_f16x2(p_lop3_and_or(w[c], 0x00F000F0u, 0x64006400u), zoff16), s2_16);
-                        const uint32_t d26 = p_mul_f16x2(p_sub_f16x2(p_lop3_and_or(w8, 0x000F000Fu, 0x64006400u), zoff), s2);
-                        const uint32_t d37 = p_mul_f16x2(p_sub_f16x2(p_lop3_and_or(w8, 0x00F000F0u, 0x64006400u), zoff16), s2_16);
-                        const uint32_t o01 = p_prmt(d04, d15, 0x5410), o45 = p_prmt(d04, d15, 0x7632);
-                        const uint32_t o23 = p_prmt(d26, d37, 0x5410), o67 = p_prmt(d26, d37, 0x7632);
+                        const uint32_t d04 = f16x2_mul(f16x2_sub(lop3_and_or(w[c], 0x000F000Fu, 0x64006400u), zoff), s2);
+                        const uint32_t d15 = f16x2_mul(f16x2_sub(lop3_and_or(w[c], 0x00F000F0u, 0x64006400u), zoff16), s2_16);
+                        const uint32_t d26 = f16x2_mul(f16x2_sub(lop3_and_or(w8, 0x000F000Fu, 0x64006400u), zoff), s2);
+                        const uint32_t d37 = f16x2_mul(f16x2_sub(lop3_and_or(w8, 0x00F000F0u, 0x64006400u), zoff16), s2_16);
+                        const uint32_t o01 = prmt(d04, d15, 0x5410), o45 = prmt(d04, d15, 0x7632);
+                        const uint32_t o23 = prmt(d26, d37, 0x5410), o67 = prmt(d26, d37, 0x7632);
                         const uint32_t addr = dst + ((((uint32_t)c) ^ swz) << 4);
                         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(o01), "r"(o23), "r"(o45), "r"(o67) : "memory");
                     }
@@ -333,9 +308,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             float f[4];
 #pragma unroll
                             for (int b = 0; b < 4; ++b)  // (q - zero) exactly, times the scale exactly (8 x 8 bits)
-                                f[b] = __fmul_rn(__fsub_rn(__uint_as_float(p_prmt(u, 0x4B000000u, 0x7650u + (uint32_t)b)), zf), sf);
-                            o[2 * h] = p_pack_f16x2(f[0], f[1]);  // the one rounding
-                            o[2 * h + 1] = p_pack_f16x2(f[2], f[3]);
+                                f[b] = __fmul_rn(__fsub_rn(__uint_as_float(prmt(u, 0x4B000000u, 0x7650u + (uint32_t)b)), zf), sf);
+                            o[2 * h] = pack_f16x2_rn(f[0], f[1]);  // the one rounding
+                            o[2 * h + 1] = pack_f16x2_rn(f[2], f[3]);
                         }
                         const uint32_t addr = dst + ((((uint32_t)c) ^ swz) << 4);
                         asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
@@ -454,6 +429,13 @@ bool prefill_supported(int M, int N, int K, int bits, int g) {
     // one tile of rows: only when the feature tiles alone fill most of the SMs (no split-K here; the
     // split-K kernel takes the layers with few output features)
     return M > 32 && (N + PM - 1) / PM >= 100;
+}
+
+void prefill_plan(int M, int N, int *bn, long long *tiles, int *ctas) {
+    const int sms = prefill_sm_count();
+    *bn = prefill_bn(M, N, sms);
+    *tiles = (long long)((N + PM - 1) / PM) * ((M + *bn - 1) / *bn);
+    *ctas = (int)(*tiles < sms ? *tiles : sms);
 }
 
 size_t prefill_scratch_bytes(int M, int K) { return round_up((size_t)M * K * 2, 256) + round_up((size_t)M * 4, 256); }

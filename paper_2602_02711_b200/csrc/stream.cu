@@ -65,38 +65,10 @@ constexpr int kClusterMaxSteps = 1600;                     // layers of up to th
 // Shared memory for the stage ring, KB: two 8-row CTAs share an SM, a 16-row CTA has it alone.
 __host__ __device__ constexpr int stage_budget_kb(int nt) { return nt == 1 ? 92 : (nt == 2 ? 100 : 136); }
 
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                               uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv) {
-    uint32_t r;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(mask), "r"(orv));  // (a & b) | c
-    return r;
-}
 
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t r;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-    return r;
-}
 
-__device__ __forceinline__ uint32_t bf16x2_sub(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
-}
 
-__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
@@ -118,8 +90,6 @@ __device__ __forceinline__ int atom_add_acq_rel(int32_t *p, int v) {
     asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
     return old;
 }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // Fragment row g of a 16-row tile holds tile row tile_row_of(g) (and that + 8): rows 0,4,1,5,...
 // so that the eight lanes of one shared-memory phase (two values of g, four 16-byte chunks each)
@@ -1058,7 +1028,14 @@ dmr_status_t launch_stream_nt(const CUtensorMap &wmap, const CUtensorMap &xmap, 
 
 size_t stream_scratch_bytes(int N) {
     const size_t groups = (size_t)(N + kTileRows - 1) / kTileRows;
-    return groups * kCounterStride * sizeof(int32_t) + (size_t)kMaxStreamCtas * 2 * 16 * kTileRows * sizeof(float);
+    return kStreamPartialBytes + groups * kCounterStride * sizeof(int32_t);
+}
+
+void stream_plan(int M, int N, int K, int bits, int *tiles, long long *steps, int *cluster) {
+    const int step_k = 1024 / bits;
+    *tiles = M <= 8 ? 1 : (M <= 16 ? 2 : 4);
+    *steps = (long long)((N + kTileRows - 1) / kTileRows) * ((K + step_k - 1) / step_k);
+    *cluster = (cluster_enabled() && *steps <= (bits == 16 ? kClusterMaxStepsDense : kClusterMaxSteps)) ? cluster_size(*tiles) : 0;
 }
 
 bool stream_supported(int M, int N, int K, int bits /*16 = bf16 weights*/, int g) {
@@ -1083,8 +1060,11 @@ dmr_status_t launch_stream(const uint16_t *X, int M, RowSel sel, const void *wei
     a.zeros = zeros;
     a.Y = Y;
     const size_t groups = (size_t)(N + kTileRows - 1) / kTileRows;
-    a.counters = reinterpret_cast<int32_t *>(scratch);
-    a.partial = reinterpret_cast<float *>(reinterpret_cast<char *>(scratch) + groups * kCounterStride * sizeof(int32_t));
+    // The partial sums come first (a fixed size) and the counters after them, so that a counter's address never
+    // depends on N: layers of different widths can share one scratch area without one layer's partial sums
+    // landing on words that another layer needs to find zero.
+    a.partial = reinterpret_cast<float *>(scratch);
+    a.counters = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(scratch) + kStreamPartialBytes);
     a.status = status;
     a.M = M;
     a.coff = sel.offset;
