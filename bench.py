@@ -34,10 +34,29 @@ METRIC = "low-bit linear: decode weight GB/s vs HBM peak; prefill TFLOP/s vs bf1
 WORKLOAD = "decode sweep, 7B-class layer (qkv, o, gate_up, down), M in {1,8,16}, INT4 g=128"
 DECODE_MS = (1, 8, 16)
 BITS, GROUP = 4, 128
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of decode_stream_kernel, mean of the four 7B-class
-# linears at M = 1 (ncu capture summarised in profiles/decode_stream_kernel_int4_g128_7b_M1.txt)
-DECODE_TRAFFIC_BYTES_PER_LAUNCH = 26.56e6
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of decode_w4_kernel, mean of the four 7B-class
+# linears at M = 1 (ncu capture summarised in profiles/decode_w4_kernel_int4_g128_7b_M1.txt)
+DECODE_TRAFFIC_BYTES_PER_LAUNCH = 26.55e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def emit_section(name, obj):
+    """Full per-section results go out as a line of their own (and into gpurun_out/ when that folder exists); the
+    final line of the run only carries short summaries."""
+    line = json.dumps({"section": name, "results": obj})
+    print(line, flush=True)
+    d = os.path.join(ROOT, "gpurun_out")
+    if os.path.isdir(d):
+        try:
+            with open(os.path.join(d, "bench_sections.jsonl"), "a") as f:
+                f.write(line + "\n")
+        except OSError:
+            pass
+
+
+def copies_beyond_l2(nbytes, l2_bytes, least=3):
+    """How many independent copies of a tensor set to rotate over so that more than 3 x L2 lies between two uses."""
+    return max(least, int(np.ceil(3.0 * l2_bytes / max(nbytes, 1))) + 1)
 
 
 def load_peaks():
@@ -220,7 +239,7 @@ def run_ours(args):
     peaks = load_peaks()
     fmt = QFormat(BITS, GROUP)
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost", "kl"}
+    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost", "kl", "crossover"}
 
     def bf16_dev(bits_np):
         return torch.from_numpy(bits_np.view(np.int16)).view(torch.bfloat16).to(dev)
@@ -303,28 +322,39 @@ def run_ours(args):
             "gpu_launches": n_launch,
             "roofline": {"bound": "hbm", "achieved": per_gpu, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": per_gpu / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_BYTES_PER_LAUNCH,
-                         "kernel": "decode_stream_kernel", "peak_source": peaks["_source"],
+                         "kernel": "decode_w4_kernel", "peak_source": peaks["_source"],
                          "us_per_launch": seconds / n_launch * 1e6,
                          "algorithmic_bytes_per_launch": step_bytes / launches_per_step},
         })
 
-        # per-shape decode numbers (same rotation, one shape at a time)
+        # per-shape decode numbers: each shape alone, over enough copies of its own that 3 x L2 lies between two uses
+        # of a copy; one CUDA graph holds one round over the copies (a chain of launches, as in a decoder)
         if "decode" in sections and rank == 0:
             per = {}
-            for name in names:
+            for i, name in enumerate(names):
+                N, K = shapes[name]
+                b = layers[0][name].weight_bytes()
+                nc = copies_beyond_l2(b, l2_bytes)
+                qs = [layers[c][name] for c in range(min(nc, copies))]
+                for c in range(len(qs), nc):
+                    g = torch.Generator(device=dev)
+                    g.manual_seed(5000 + 100 * i + c)
+                    W = (torch.randn((N, K), generator=g, device=dev, dtype=torch.float32) * inputs.WEIGHT_SIGMA).to(torch.bfloat16)
+                    qs.append(dmr.dmr_quantize(W, fmt))
+                    del W
                 for M in DECODE_MS:
-                    gs = []
-                    for c in range(copies):
-                        g = torch.cuda.CUDAGraph()
-                        with torch.cuda.graph(g, stream=stream):
-                            dmr.dmr_lowbit_linear(X[(name, M)], layers[c][name], OUT_BF16, Y=Y[(name, M)], workspace=ws)
-                        gs.append(g)
-                    reps = 40 * copies
-                    sec = time_graph_replays(gs, reps, copies, torch)
-                    b = layers[0][name].weight_bytes()
-                    per[f"{name}_M{M}"] = {"us": sec / reps * 1e6, "gbs": b * reps / sec / 1e9,
-                                          "frac_hbm": b * reps / sec / 1e9 / peaks["hbm_gbs"]}
-            result["decode_per_shape"] = per
+                    for c in range(nc):
+                        dmr.dmr_lowbit_linear(X[(name, M)], qs[c], OUT_BF16, Y=Y[(name, M)], workspace=ws)
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        for c in range(nc):
+                            dmr.dmr_lowbit_linear(X[(name, M)], qs[c], OUT_BF16, Y=Y[(name, M)], workspace=ws)
+                    rounds = max(3, 160 // nc)
+                    sec = time_graph_replays([g], rounds, 2, torch) / (rounds * nc)
+                    per[f"{name}_M{M}"] = {"us": sec * 1e6, "gbs": b / sec / 1e9, "frac_hbm": b / sec / 1e9 / peaks["hbm_gbs"], "copies": nc}
+                del qs
+            emit_section("decode_per_shape", per)
+            result["decode_frac_hbm"] = {k: round(v["frac_hbm"], 3) for k, v in per.items()}
 
         # end-to-end: host activations in, host outputs back, through the host-buffer entry point
         if "e2e" in sections:
@@ -357,21 +387,35 @@ def run_ours(args):
                              "note": "weights resident on the device; activations copied in and outputs copied "
                                      "back every call through dmr_lowbit_linear_host"}
 
-        extra = run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copies, stream)
+        extra = run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, l2_bytes, stream)
         result.update(extra)
 
     if rank == 0:
         if "cpu" in sections and world >= 1:
             v, cores, sample = oracle_cpu_baseline()
             result["cpu_baseline"] = {"value": v, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample}
+        # the run's records keep the end of the output: a short summary of every section goes last
+        summary = {}
+        if "roofline_prefill" in result:
+            rp = result["roofline_prefill"]
+            summary["prefill_frac_bf16_burst_by_M"] = rp["frac_by_M"]
+            summary["prefill_M8192"] = {"tflops": round(rp["achieved"], 1), "us": round(rp["us"], 1)}
+        if "routed" in result:
+            summary["routed_14b_M64"] = {"layer_us": round(result["routed"]["layer_us"], 1), "frac_hbm": round(result["routed"]["frac_hbm"], 3)}
+        for key in ("crossover_32b", "dense_decode_frac_hbm", "layer_cost_7b", "stepwise_kl"):
+            if key in result:
+                summary[key] = result.pop(key)
+        result["summary"] = summary
         print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()
 
 
-def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copies, stream):
-    """Prefill, routed, dense and quantize numbers (rank 0 only; not part of the timed headline)."""
-    from paper_2602_02711_b200 import OUT_BF16
+def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, l2_bytes, stream):
+    """Prefill, routed, dense, crossover, cost-model, KL and quantize numbers (rank 0 only; not part of the timed
+    headline).  Every section prints its full table as a line of its own and returns a short summary."""
+    from paper_2602_02711_b200 import OUT_BF16, QFormat as QF, cost
+    from paper_2602_02711_b200.binding import OP_LOWBIT, OP_DENSE
     out = {}
     if rank != 0:
         return out
@@ -398,6 +442,19 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) * 1e-3 / reps
 
+    def time_rotating(call, ncopy, reps):
+        """Seconds per call of call(c), c = 0 .. ncopy - 1 visited in rotation: one CUDA graph holds one round over
+        all copies, so the figure is device time and every call meets weights that left the L2 long ago."""
+        for c in range(ncopy):
+            call(c)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for c in range(ncopy):
+                call(c)
+        rounds = max(2, int(np.ceil(reps / ncopy)))
+        return timeit(g.replay, reps=rounds, warm=2) / ncopy
+
     if "prefill" in sections:
         pre = {}
         for name, (N, K) in inputs.LAYER_7B.items():
@@ -408,86 +465,74 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
                 X = randx(M, K, M)
                 Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
                 ws = dmr.new_workspace(0, M, N, K, fmt, dev)
-                t = timeit(lambda: dmr.dmr_lowbit_linear(X, q, OUT_BF16, Y=Y, workspace=ws), reps=5, warm=2)
+                t = timeit(lambda: dmr.dmr_lowbit_linear(X, q, OUT_BF16, Y=Y, workspace=ws), reps=20, warm=3)
                 tf = 2.0 * M * N * K / t / 1e12
                 pre[f"{name}_M{M}"] = {"us": t * 1e6, "tflops": tf, "frac_bf16_burst": tf / peaks["bf16_tflops"],
-                                       "frac_bf16_sustained": tf / peaks["bf16_tflops_sustained"]}
+                                       "frac_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+                                       "kernel": dmr.dmr_describe_dispatch(OP_LOWBIT, M, N, K, fmt)}
                 del X, Y
             del q
-        out["prefill"] = pre
+        emit_section("prefill", pre)
+        per_m = {}
+        for M in (512, 2048, 8192):
+            fl = sum(2.0 * M * N * K for N, K in inputs.LAYER_7B.values())
+            tt = sum(pre[f"{name}_M{M}"]["us"] for name in inputs.LAYER_7B) * 1e-6
+            per_m[M] = {"tflops": fl / tt / 1e12, "us": tt * 1e6}
         # all four linears at M = 8192 as one figure for the tensor-core roofline
-        fl = sum(2.0 * 8192 * N * K for N, K in inputs.LAYER_7B.values())
-        tt = sum(pre[f"{name}_M8192"]["us"] for name in inputs.LAYER_7B) * 1e-6
-        out["roofline_prefill"] = {"bound": "tensor", "achieved": fl / tt / 1e12, "peak": peaks["bf16_tflops"],
-                                   "unit": "TFLOP/s", "frac": fl / tt / 1e12 / peaks["bf16_tflops"], "traffic": None,
-                                   "kernel": "prefill_kernel", "peak_source": peaks["_source"] + " (burst)",
-                                   "workload": "7B-class layer, four linears, M=8192, INT4 g=128, bf16 out"}
+        out["roofline_prefill"] = {"bound": "tensor", "achieved": per_m[8192]["tflops"], "peak": peaks["bf16_tflops"],
+                                   "unit": "TFLOP/s", "frac": per_m[8192]["tflops"] / peaks["bf16_tflops"], "traffic": None,
+                                   "us": per_m[8192]["us"], "kernel": "prefill_kernel", "peak_source": peaks["_source"] + " (burst)",
+                                   "frac_by_M": {str(M): round(v["tflops"] / peaks["bf16_tflops"], 3) for M, v in per_m.items()},
+                                   "workload": "7B-class layer, four linears, INT4 g=128, bf16 out; headline figure at M=8192"}
 
     if "routed" in sections:
         M = 64
         tot_t, tot_b, per = 0.0, 0.0, {}
         for name, (N, K) in inputs.LAYER_14B.items():
-            # rotate over copies so that neither weight set is served from L2
-            nc = 3
+            # enough copies of both weight sets that neither is served from the L2
+            nc = copies_beyond_l2(N * K * 2.5234, l2_bytes)
             Ws = [randw(N, K, 31 + c) for c in range(nc)]
             qs = [dmr.dmr_quantize(w, fmt) for w in Ws]
             X = randx(M, K, 7)
             mask = torch.from_numpy(inputs.precision_mask(M, 0.3, seed=0)).to(dev)
             Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
             ws = dmr.new_workspace(2, M, N, K, fmt, dev)
-            # one CUDA graph per weight copy (a routed call is several launches: partition, gathers, the two
-            # halves), replayed in rotation, so that the figure is device time and not Python launch overhead
-            for c in range(nc):
-                dmr.dmr_routed_linear(X, mask, Ws[c], qs[c], OUT_BF16, Y=Y, workspace=ws)
-            torch.cuda.synchronize()
-            graphs = []
-            for c in range(nc):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=stream):
-                    dmr.dmr_routed_linear(X, mask, Ws[c], qs[c], OUT_BF16, Y=Y, workspace=ws)
-                graphs.append(g)
-            state = {"i": 0}
-
-            def call():
-                state["i"] += 1
-                graphs[state["i"] % nc].replay()
-
-            t = timeit(call, reps=30, warm=3)
+            t = time_rotating(lambda c: dmr.dmr_routed_linear(X, mask, Ws[c], qs[c], OUT_BF16, Y=Y, workspace=ws), nc, reps=30)
             b = N * K * 2 + qs[0].weight_bytes()
-            per[name] = {"us": t * 1e6, "gbs": b / t / 1e9, "frac_hbm": b / t / 1e9 / peaks["hbm_gbs"]}
+            per[name] = {"us": t * 1e6, "gbs": b / t / 1e9, "frac_hbm": b / t / 1e9 / peaks["hbm_gbs"], "copies": nc}
             tot_t += t
             tot_b += b
             del Ws, qs
+        emit_section("routed", per)
         out["routed"] = {"layer_us": tot_t * 1e6, "gbs": tot_b / tot_t / 1e9, "frac_hbm": tot_b / tot_t / 1e9 / peaks["hbm_gbs"],
-                         "workload": "14B-class layer, 7 linears, M=64, mask~Bernoulli(0.3)", "per_linear": per}
+                         "workload": "14B-class layer, 7 linears, M=64, mask~Bernoulli(0.3)",
+                         "us": {k: round(v["us"], 1) for k, v in per.items()}}
 
     if "dense" in sections:
         den = {}
         for name, (N, K) in inputs.LAYER_7B.items():
-            Ws = [randw(N, K, 41 + c) for c in range(3)]
+            nc = copies_beyond_l2(N * K * 2, l2_bytes)
+            Ws = [randw(N, K, 41 + c) for c in range(nc)]
             for M in (1, 16):
                 X = randx(M, K, 3)
                 Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
                 ws = dmr.new_workspace(1, M, N, K, fmt, dev)
-                state = {"i": 0}
-
-                def call():
-                    state["i"] += 1
-                    dmr.dmr_dense_linear(X, Ws[state["i"] % 3], OUT_BF16, Y=Y, workspace=ws)
-
-                t = timeit(call, reps=30)
-                den[f"{name}_M{M}"] = {"us": t * 1e6, "gbs": N * K * 2 / t / 1e9, "frac_hbm": N * K * 2 / t / 1e9 / peaks["hbm_gbs"]}
+                t = time_rotating(lambda c: dmr.dmr_dense_linear(X, Ws[c], OUT_BF16, Y=Y, workspace=ws), nc, reps=40)
+                den[f"{name}_M{M}"] = {"us": t * 1e6, "gbs": N * K * 2 / t / 1e9, "frac_hbm": N * K * 2 / t / 1e9 / peaks["hbm_gbs"],
+                                       "copies": nc}
             del Ws
-        out["dense_decode"] = den
+        emit_section("dense_decode", den)
+        out["dense_decode_frac_hbm"] = {k: round(v["frac_hbm"], 3) for k, v in den.items()}
 
     if "layer_cost" in sections:
         # Per-token decode cost of one 7B-class layer at bf16 (T_high) and at INT4 g=128 (T_low): the four
         # linears chained in one CUDA graph, weights rotated over copies so that they come from HBM.  The
-        # latency-based cost of the paper (Sec. 4.3, cost C = T_router N_steps + T_high N_high + T_low N_low)
-        # then gives the relative cost of a routed run at high-precision budget rho, router cost aside:
-        # C(rho) / C(all bf16) = rho + (1 - rho) T_low / T_high.
+        # latency-based cost of the paper (Sec. 4.3, C = T_router N_steps + T_high N_high + T_low N_low) then
+        # gives the relative cost of a routed run at high-precision budget rho; the router's own time is left
+        # out (no router is built here), which the output says.
         lc = {}
-        ncopy = 3
+        layer_bf16 = sum(N * K * 2 for N, K in inputs.LAYER_7B.values())
+        ncopy = copies_beyond_l2(layer_bf16, l2_bytes)
         Ws = [{n: randw(N, K, 71 + 7 * c + i) for i, (n, (N, K)) in enumerate(inputs.LAYER_7B.items())} for c in range(ncopy)]
         Qs = [{n: dmr.dmr_quantize(w, fmt) for n, w in layer.items()} for layer in Ws]
         for M in (1, 16):
@@ -495,58 +540,61 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
             Ys = {n: torch.empty((M, N), dtype=torch.bfloat16, device=dev) for n, (N, K) in inputs.LAYER_7B.items()}
             wsd = dmr.new_workspace(1, M, 22016, 11008, fmt, dev)
             wsl = dmr.new_workspace(0, M, 22016, 11008, fmt, dev)
-            times = {}
-            for kind in ("bf16", "int4"):
-                graphs = []
-                for c in range(ncopy):
-                    g = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(g, stream=stream):
-                        for n in inputs.LAYER_7B:
-                            if kind == "bf16":
-                                dmr.dmr_dense_linear(Xs[n], Ws[c][n], OUT_BF16, Y=Ys[n], workspace=wsd)
-                            else:
-                                dmr.dmr_lowbit_linear(Xs[n], Qs[c][n], OUT_BF16, Y=Ys[n], workspace=wsl)
-                    graphs.append(g)
-                state = {"i": 0}
 
-                def call():
-                    state["i"] += 1
-                    graphs[state["i"] % ncopy].replay()
+            def layer_call(kind):
+                def call(c):
+                    for n in inputs.LAYER_7B:
+                        if kind == "bf16":
+                            dmr.dmr_dense_linear(Xs[n], Ws[c][n], OUT_BF16, Y=Ys[n], workspace=wsd)
+                        else:
+                            dmr.dmr_lowbit_linear(Xs[n], Qs[c][n], OUT_BF16, Y=Ys[n], workspace=wsl)
+                return call
 
-                times[kind] = timeit(call, reps=60)
-            ratio = times["int4"] / times["bf16"]
-            lc[f"M{M}"] = {"t_high_us_per_layer": times["bf16"] * 1e6, "t_low_us_per_layer": times["int4"] * 1e6,
-                           "t_high_over_t_low": 1.0 / ratio,
-                           "relative_cost_at_budget": {f"rho={r}": r + (1 - r) * ratio for r in (0.2, 0.4, 0.7)}}
+            t_high = time_rotating(layer_call("bf16"), ncopy, reps=60)
+            t_low = time_rotating(layer_call("int4"), ncopy, reps=60)
+            lc[f"M{M}"] = {"t_high_us_per_layer": t_high * 1e6, "t_low_us_per_layer": t_low * 1e6,
+                           "t_high_over_t_low": t_high / t_low, "t_router": "excluded (no router in this library)",
+                           "relative_cost_at_budget": {f"rho={r}": cost.relative_cost_at_budget(r, t_high, t_low) for r in (0.2, 0.4, 0.7)}}
         del Ws, Qs
-        out["layer_cost_7b"] = lc
+        emit_section("layer_cost_7b", lc)
+        out["layer_cost_7b"] = {k: {"t_high_us": round(v["t_high_us_per_layer"], 1), "t_low_us": round(v["t_low_us_per_layer"], 1),
+                                    "ratio": round(v["t_high_over_t_low"], 2)} for k, v in lc.items()}
 
     if "crossover" in sections:
-        # 32B-class gate and down linears, INT4 g=64 and INT8 per-channel, M = 1 .. 256, 1 % outlier channels x20:
-        # where the library's dispatch (streaming kernel up to 32 rows, tensor-core kernels above) stands.
-        # The streaming family at larger M is timed by separate runs with DMR_DECODE_MAX_M=256.
-        from paper_2602_02711_b200 import QFormat as QF
+        # 32B-class gate and down linears, INT4 g=64 and INT8 per-channel, M = 1 .. 256, 1 % outlier channels x20,
+        # with the library's default dispatch (decode kernels up to 32 rows, tensor-core kernels above): where
+        # the bandwidth-bound family hands over to the compute-bound one.  Two weight copies exceed 3 x L2 for INT8
+        # (141 MB each) and come close for INT4 g64 (77 MB each; three copies are used).
         cx = {"dispatch": f"DMR_DECODE_MAX_M={os.environ.get('DMR_DECODE_MAX_M', '32')}"}
+        summary = {}
         for lname, (N, K) in inputs.LAYER_32B.items():
             for fname, f5 in (("int4_g64", QF(4, 64)), ("int8_pc", QF(8, 0))):
-                Ws = [randw(N, K, 61 + c) for c in range(2)]
-                qs = [dmr.dmr_quantize(w, f5) for w in Ws]
-                del Ws
+                wb = N * K * f5.bits // 8
+                nc = copies_beyond_l2(wb, l2_bytes, least=2)
+                qs = []
+                for c in range(nc):
+                    w = randw(N, K, 61 + c)
+                    qs.append(dmr.dmr_quantize(w, f5))
+                    del w
+                best = None
                 for M in (1, 2, 4, 8, 16, 32, 64, 128, 256):
                     X = torch.from_numpy(inputs.activations(M, K, seed=5, index=M, outlier_frac=0.01).view(np.int16)).view(torch.bfloat16).to(dev)
                     Y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
                     ws = dmr.new_workspace(0, M, N, K, f5, dev)
-                    state = {"i": 0}
-
-                    def call():
-                        state["i"] += 1
-                        dmr.dmr_lowbit_linear(X, qs[state["i"] % 2], OUT_BF16, Y=Y, workspace=ws)
-
-                    t = timeit(call, reps=20)
+                    t = time_rotating(lambda c: dmr.dmr_lowbit_linear(X, qs[c], OUT_BF16, Y=Y, workspace=ws), nc, reps=12)
                     b = qs[0].weight_bytes()
-                    cx[f"{lname}_{fname}_M{M}"] = {"us": t * 1e6, "gbs": b / t / 1e9, "tflops": 2.0 * M * N * K / t / 1e12}
+                    kern = dmr.dmr_describe_dispatch(OP_LOWBIT, M, N, K, f5)["kernel"]
+                    cx[f"{lname}_{fname}_M{M}"] = {"us": t * 1e6, "gbs": b / t / 1e9, "tflops": 2.0 * M * N * K / t / 1e12, "kernel": kern}
+                    if kern in ("decode_w4", "stream"):
+                        best = M
+                summary[f"{lname}_{fname}"] = {
+                    "M1_frac_hbm": round(cx[f"{lname}_{fname}_M1"]["gbs"] / peaks["hbm_gbs"], 3),
+                    "M16_frac_hbm": round(cx[f"{lname}_{fname}_M16"]["gbs"] / peaks["hbm_gbs"], 3),
+                    "M256_tflops": round(cx[f"{lname}_{fname}_M256"]["tflops"], 1),
+                    "last_M_on_decode_kernels": best}
                 del qs
-        out["crossover_32b"] = cx
+        emit_section("crossover_32b", cx)
+        out["crossover_32b"] = summary
 
     if "kl" in sections:
         # Step-wise KL divergence: two [T][V] bf16 logit tensors (1.24 GB, far beyond the L2) read once.
@@ -558,9 +606,10 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
         offs = torch.from_numpy(inputs.step_offsets(T, 12, seed=3)).to(dev)
         t = timeit(lambda: dmr.dmr_stepwise_kl(hi, lo, offs), reps=10, warm=3)
         b = 2.0 * T * V * 2
-        out["stepwise_kl"] = {"us": t * 1e6, "gbs": b / t / 1e9, "frac_hbm": b / t / 1e9 / peaks["hbm_gbs"],
-                              "tokens_per_s": T / t,
-                              "workload": f"{T} action tokens x {V} logits, bf16, two models, {int(offs.numel()) - 1} steps"}
+        kl = {"us": t * 1e6, "gbs": b / t / 1e9, "frac_hbm": b / t / 1e9 / peaks["hbm_gbs"], "tokens_per_s": T / t,
+              "workload": f"{T} action tokens x {V} logits, bf16, two models, {int(offs.numel()) - 1} steps"}
+        emit_section("stepwise_kl", kl)
+        out["stepwise_kl"] = {"us": round(kl["us"], 1), "frac_hbm": round(kl["frac_hbm"], 3)}
         del hi, lo
 
     if "quantize" in sections:
@@ -570,7 +619,8 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, copi
             t = timeit(lambda: dmr.dmr_quantize(W, fmt, check=False), reps=5, warm=2)
             qz[name] = {"us": t * 1e6, "gweights_per_s": N * K / t / 1e9}
             del W
-        out["quantize"] = qz
+        emit_section("quantize", qz)
+        out["quantize_us"] = {k: round(v["us"], 1) for k, v in qz.items()}
     return out
 
 
@@ -580,7 +630,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost,kl")
+    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost,kl (default: all; none = headline only)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
