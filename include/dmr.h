@@ -28,6 +28,12 @@
  * The library allocates no device memory.  `stream` is a cudaStream_t passed as void*; all work
  * is enqueued on it and no call synchronises the host.  Argument errors are reported before
  * anything is launched.  Pointers must be 16-byte aligned.
+ *
+ * Threads.  Every entry point may be called from several host threads at once as long as calls that can
+ * overlap on the GPU use different workspaces (and outputs).  The library's own host state - a cache of TMA
+ * tensor maps keyed by address and shape, the per-kernel set-up flags, the launch counter - is guarded
+ * inside; dmr_routed_linear calls of one process take turns while they enqueue (they share one helper stream
+ * per device), which costs host time only.  dmr_last_cuda_error reports the last failure of any thread.
  */
 #ifndef DMR_H_
 #define DMR_H_
@@ -90,7 +96,8 @@ size_t dmr_workspace_bytes(dmr_op_t op, int M, int N, int K, dmr_qformat_t f);
 dmr_status_t dmr_quantize(const void *W_bf16, int N, int K, dmr_qformat_t f, void *qweight,
                           void *scales, void *zeros, int32_t *dev_status, void *stream);
 
-/* Test utility: W_out[n][k] = scale * (code - zero), as fp32 (exact) or bf16 (nearest). */
+/* Test utility: W_out[n][k] = scale * (code - zero), as fp32 (exact) or bf16 (nearest): the weights the
+ * low-precision model of Sec. 5 / App. "Quantization Detail" computes with, written out. */
 dmr_status_t dmr_dequantize(const void *qweight, const void *scales, const void *zeros, int N,
                             int K, dmr_qformat_t f, void *W_out, dmr_out_t out, void *stream);
 
@@ -129,7 +136,9 @@ dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, c
                                size_t workspace_bytes, void *stream);
 
 /*
- * Stable partition of step indices by mask (the split that dmr_routed_linear performs first).
+ * Stable partition of step indices by mask (the split that dmr_routed_linear performs first): the per-step
+ * routing index r_t of Sec. 3, Eq. 1, turned into the two lists of steps each precision serves; mask != 0
+ * marks the steps whose router score reached the threshold of Sec. 4.2 "Inference-time calibration".
  * idx_high / idx_low: int32 [M] each; counts: int32 [2] = {n_high, n_low}.  All on the device.
  */
 dmr_status_t dmr_route_partition(const uint8_t *mask, int M, int32_t *idx_high, int32_t *idx_low,
@@ -193,6 +202,33 @@ dmr_status_t dmr_lowbit_linear_noalloc(const void *X_bf16, int M, const void *qw
 dmr_status_t dmr_stepwise_kl(const void *logits_high, const void *logits_low, dmr_out_t dtype, int T,
                              int V, const int32_t *step_offsets, int S, float *kl_token, float *kl_step,
                              void *stream);
+
+/*
+ * Inference-time calibration of the router (Sec. 4.2 "Inference-time calibration"): for a high-precision budget
+ * rho the threshold is tau(rho) = Quantile(D_cal, 1 - rho) over the router's scores on a calibration pool (the
+ * paper uses rho in {0.20, 0.40, 0.70}), and a step goes to the high-precision model when its score p_t >= tau.
+ *   dmr_router_calibrate: cal_scores device fp32 [n], finite, 1 <= n <= 65536 (more: DMR_ERR_UNSUPPORTED);
+ *       0 <= rho <= 1; tau: device, THREE doubles, 16-byte aligned - tau[0] receives the threshold, tau[1..2] are
+ *       scratch.  Quantile rule (the paper names none): linear interpolation between order statistics,
+ *       x_(lo) + (h - lo)(x_(lo+1) - x_(lo)) with h = (n - 1)(1 - rho), lo = floor(h), in binary64.
+ *   dmr_router_mask: scores device fp32 [M] -> mask device uint8 [M], mask[m] = (scores[m] >= tau[0]) ? 1 : 0, the
+ *       mask dmr_routed_linear takes (1 = high precision).  tau is read on the device: no host round trip between
+ *       calibration, masking and the routed layer.  M = 0 is a no-op.
+ * Errors: DMR_ERR_INVALID_ARG (null pointer, n < 1, M < 0, rho outside [0, 1]), DMR_ERR_ALIGNMENT, DMR_ERR_CUDA.
+ */
+dmr_status_t dmr_router_calibrate(const float *cal_scores, int n, double rho, double *tau, void *stream);
+dmr_status_t dmr_router_mask(const float *scores, int M, const double *tau, uint8_t *mask, void *stream);
+
+/*
+ * Self-test of the bounded waits (no counterpart in the paper).  Every wait inside the kernels gives up after a
+ * fixed number of polls, writes DMR_ERR_TIMEOUT to the workspace's status word and lets the kernel finish, so a
+ * copy that never lands cannot hang the GPU.  This call launches one warp that waits - with the limit lowered
+ * to a thousand polls - on a barrier nothing ever arrives at.  Afterwards dmr_workspace_status(workspace)
+ * returns DMR_ERR_TIMEOUT and the second int32 of the workspace holds 2 (the kernel ran to its end).  The
+ * caller clears the first 256 bytes of the workspace before using it for other calls again.
+ * workspace: at least 256 bytes, zero-filled.
+ */
+dmr_status_t dmr_selftest_wait_timeout(void *workspace, size_t workspace_bytes, void *stream);
 
 /* Reads the status word a previous call may have set in `workspace` (DMR_OK or DMR_ERR_TIMEOUT).
  * Synchronises `stream`. */

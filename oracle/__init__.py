@@ -234,3 +234,26 @@ def stepwise_kl(logits_high: np.ndarray, logits_low: np.ndarray, step_offsets):
         seg = kl_token[off[s]:off[s + 1]]
         kl_step[s] = seg.mean() if len(seg) else 0.0
     return kl_step, kl_token
+
+
+def router_threshold(cal_scores, rho: float) -> float:
+    """tau(rho) = Quantile(D_cal, 1 - rho) (Sec. 4.2 "Inference-time calibration"), in float64.
+
+    The paper names no quantile rule; the reading taken is linear interpolation between order statistics: sort
+    the scores ascending, h = (n - 1)(1 - rho), lo = floor(h), tau = x[lo] + (h - lo) * (x[lo + 1] - x[lo])
+    (x[n - 1] when lo is the last index). Scores are widened exactly to float64 first.
+    """
+    x = np.sort(np.asarray(cal_scores).astype(np.float64))
+    n = len(x)
+    if n < 1 or not (0.0 <= rho <= 1.0):
+        raise ValueError("need at least one score and 0 <= rho <= 1")
+    h = float(n - 1) * (1.0 - float(rho))
+    lo = min(int(np.floor(h)), n - 1)
+    hi = min(lo + 1, n - 1)
+    gamma = h - float(lo)
+    return float(x[lo] + gamma * (x[hi] - x[lo]))
+
+
+def router_mask(scores, tau: float) -> np.ndarray:
+    """mask[m] = 1 where the step's router score reaches the threshold (p_t >= tau: high precision), else 0."""
+    return (np.asarray(scores).astype(np.float64) >= float(tau)).astype(np.uint8)

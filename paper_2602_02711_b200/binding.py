@@ -76,6 +76,12 @@ def lib() -> ctypes.CDLL:
     L.dmr_noalloc_max_n.restype = i32
     L.dmr_lowbit_linear_noalloc.restype = i32
     L.dmr_lowbit_linear_noalloc.argtypes = [vp, i32, vp, vp, vp, i32, i32, QFormat, vp, i32, vp]
+    L.dmr_router_calibrate.restype = i32
+    L.dmr_router_calibrate.argtypes = [vp, i32, ctypes.c_double, vp, vp]
+    L.dmr_router_mask.restype = i32
+    L.dmr_router_mask.argtypes = [vp, i32, vp, vp, vp]
+    L.dmr_selftest_wait_timeout.restype = i32
+    L.dmr_selftest_wait_timeout.argtypes = [vp, sz, vp]
     L.dmr_workspace_status.restype = i32
     L.dmr_workspace_status.argtypes = [vp, vp]
     L.dmr_describe_dispatch.restype = i32
@@ -303,3 +309,20 @@ def dmr_lowbit_linear_noalloc(X: torch.Tensor, q: QuantizedLinear, Y: torch.Tens
     _check(lib().dmr_lowbit_linear_noalloc(_ptr(X), M, _ptr(q.qweight), _ptr(q.scales), _ptr(q.zeros), q.N, K, q.fmt,
                                            _ptr(Y), out, _stream(stream)))
     return Y
+
+
+def dmr_router_calibrate(cal_scores: torch.Tensor, rho: float, stream=None) -> torch.Tensor:
+    """tau(rho) = Quantile(cal_scores, 1 - rho) on the device. Returns a float64 device tensor [3]; element 0 is tau."""
+    _dev(cal_scores, torch.float32, "cal_scores")
+    tau = torch.zeros(3, dtype=torch.float64, device=cal_scores.device)
+    _check(lib().dmr_router_calibrate(_ptr(cal_scores), cal_scores.numel(), float(rho), _ptr(tau), _stream(stream)))
+    return tau
+
+
+def dmr_router_mask(scores: torch.Tensor, tau: torch.Tensor, stream=None) -> torch.Tensor:
+    """mask[m] = 1 where scores[m] >= tau[0] (the step needs the high-precision weights), uint8 on the device."""
+    _dev(scores, torch.float32, "scores")
+    _dev(tau, torch.float64, "tau")
+    mask = torch.empty(scores.numel(), dtype=torch.uint8, device=scores.device)
+    _check(lib().dmr_router_mask(_ptr(scores), scores.numel(), _ptr(tau), _ptr(mask), _stream(stream)))
+    return mask

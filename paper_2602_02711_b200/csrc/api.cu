@@ -4,12 +4,13 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 
 namespace dmr {
-int g_last_cuda_error = 0;
-unsigned long long g_launches = 0;
+std::atomic<int> g_last_cuda_error{0};
+std::atomic<unsigned long long> g_launches{0};
 
 namespace {
 
@@ -239,7 +240,11 @@ struct SideStream {
     cudaEvent_t fork = nullptr, join = nullptr;
 };
 
-SideStream *side_stream() {
+// Routed calls of one process enqueue one at a time: the helper stream and its two events are shared per device,
+// and a second host thread recording the same events in between would tie the wrong pieces of work together.
+std::mutex g_routed_mutex;
+
+SideStream *side_stream() {  // called with g_routed_mutex held
     static SideStream per_device[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
@@ -365,6 +370,7 @@ dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, c
     if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
     cudaStream_t st = (cudaStream_t)stream;
     const Scratch ws = carve(workspace, DMR_OP_ROUTED_LINEAR, M, N, K, f);
+    std::lock_guard<std::mutex> routed_lock(g_routed_mutex);
     r = launch_route_partition(mask, M, ws.idx_high, ws.idx_low, ws.counts, st);
     if (r != DMR_OK) return r;
     const uint16_t *X = reinterpret_cast<const uint16_t *>(X_bf16);
@@ -484,6 +490,28 @@ int dmr_describe_dispatch(dmr_op_t op, int M, int N, int K, dmr_qformat_t f, cha
     stream_plan(M < kStreamChunk ? M : kStreamChunk, N, K, sbits, &tiles, &steps, &cluster);
     return snprintf(buf, buf_bytes, "stream bits=%d rows=%d steps=%lld cluster=%d chunks=%d", sbits, 8 * tiles, steps, cluster,
                     (M + kStreamChunk - 1) / kStreamChunk);
+}
+
+dmr_status_t dmr_router_calibrate(const float *cal_scores, int n, double rho, double *tau, void *stream) {
+    if (!cal_scores || !tau || n < 1) return DMR_ERR_INVALID_ARG;
+    if (!(rho >= 0.0 && rho <= 1.0)) return DMR_ERR_INVALID_ARG;
+    if (n > 65536) return DMR_ERR_UNSUPPORTED;
+    if (((uintptr_t)tau & 15u) != 0) return DMR_ERR_ALIGNMENT;  // tau[0] is the result, tau[1..2] scratch
+    return launch_router_calibrate(cal_scores, n, rho, tau, tau + 1, (cudaStream_t)stream);
+}
+
+dmr_status_t dmr_router_mask(const float *scores, int M, const double *tau, uint8_t *mask, void *stream) {
+    if (M < 0 || !tau) return DMR_ERR_INVALID_ARG;
+    if (M == 0) return DMR_OK;
+    if (!scores || !mask) return DMR_ERR_INVALID_ARG;
+    return launch_router_mask(scores, M, tau, mask, (cudaStream_t)stream);
+}
+
+dmr_status_t dmr_selftest_wait_timeout(void *workspace, size_t workspace_bytes, void *stream) {
+    if (!workspace || workspace_bytes < kWsStatusBytes) return DMR_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
+    int32_t *w = reinterpret_cast<int32_t *>(workspace);
+    return launch_wait_timeout_selftest(w, w + 1, (cudaStream_t)stream);
 }
 
 const char *dmr_status_string(dmr_status_t s) {

@@ -4,13 +4,15 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "dmr.h"
 
 namespace dmr {
 
 // ---- host-side bookkeeping -------------------------------------------------------------
-extern int g_last_cuda_error;           // last failing cudaError_t (0 if none)
-extern unsigned long long g_launches;   // kernels launched by this library in this process
+extern std::atomic<int> g_last_cuda_error;           // last failing cudaError_t (0 if none)
+extern std::atomic<unsigned long long> g_launches;   // kernels launched by this library in this process
 
 inline dmr_status_t check_launch() {
     ++g_launches;
@@ -135,5 +137,12 @@ dmr_status_t launch_route_partition(const uint8_t *mask, int M, int32_t *idx_hig
 // (bf16 or fp32), kl_step[s] = mean of kl_token over [offsets[s], offsets[s + 1]).
 dmr_status_t launch_stepwise_kl(const void *high, const void *low, bool f32, int T, int V, const int32_t *offsets, int S,
                                 float *kl_token, float *kl_step, cudaStream_t st);
+
+// Router calibration: tau = the (1 - rho) quantile of `scores` (linear interpolation, binary64); picked: 2 doubles of scratch.
+dmr_status_t launch_router_calibrate(const float *scores, int n, double rho, double *tau, double *picked, cudaStream_t st);
+dmr_status_t launch_router_mask(const float *scores, int M, const double *tau, uint8_t *mask, cudaStream_t st);
+
+// One warp waits on a barrier nobody arrives at, with a short limit: *status becomes DMR_ERR_TIMEOUT, *returned 2.
+dmr_status_t launch_wait_timeout_selftest(int32_t *status, int32_t *returned, cudaStream_t st);
 
 }  // namespace dmr

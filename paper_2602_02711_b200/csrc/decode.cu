@@ -488,17 +488,8 @@ dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
     constexpr size_t kSzBudget = 227 * 1024 - Cfg::SMEM < 36 * 1024 ? 227 * 1024 - Cfg::SMEM : 36 * 1024;
     static_assert(Cfg::SMEM <= 227 * 1024, "ring and reduction buffers exceed an SM's shared memory");
     auto kernel = decode_w4_kernel<NT, R, WPL, WARPS, D, OUT_F32>;
-    static bool configured[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
-    if (!configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(Cfg::SMEM + kSzBudget < kMinSmem ? kMinSmem : Cfg::SMEM + kSzBudget));
-        if (e != cudaSuccess) {
-            g_last_cuda_error = (int)e;
-            return DMR_ERR_CUDA;
-        }
-        configured[dev] = true;
-    }
+    if (!ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), Cfg::SMEM + kSzBudget < kMinSmem ? kMinSmem : Cfg::SMEM + kSzBudget))
+        return DMR_ERR_CUDA;
     a.tiles = (a.N + TILE - 1) / TILE;
     a.nchunks = a.K / Cfg::CHUNK_K;
     int ctas = device_sm_count();

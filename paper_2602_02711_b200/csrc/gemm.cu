@@ -345,11 +345,7 @@ dmr_status_t launch_gemm_t(const CUtensorMap &map_w, const CUtensorMap &map_x, c
     using Cfg = GemmCfg<MODE, BN>;
     dim3 grid((a.N + BM - 1) / BM, (a.M + BN - 1) / BN, splits);
     auto launch = [&](auto kernel) -> dmr_status_t {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM);
-        if (e != cudaSuccess) {
-            g_last_cuda_error = (int)e;
-            return DMR_ERR_CUDA;
-        }
+        if (!ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), Cfg::SMEM)) return DMR_ERR_CUDA;
         kernel<<<grid, Cfg::THREADS, Cfg::SMEM, st>>>(map_w, map_x, a);
         return check_launch();
     };

@@ -384,11 +384,7 @@ dmr_status_t launch_prefill_t(const CUtensorMap &map_w, const CUtensorMap &map_x
                               dmr_out_t out, cudaStream_t st) {
     using Cfg = PrefillCfg<BITS, BN>;
     auto launch = [&](auto kernel) -> dmr_status_t {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM);
-        if (e != cudaSuccess) {
-            g_last_cuda_error = (int)e;
-            return DMR_ERR_CUDA;
-        }
+        if (!ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), Cfg::SMEM)) return DMR_ERR_CUDA;
         kernel<<<grid, Cfg::THREADS, Cfg::SMEM, st>>>(map_w, map_x, a);
         return check_launch();
     };

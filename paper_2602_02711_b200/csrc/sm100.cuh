@@ -22,6 +22,9 @@ bool make_tensor_map_2d(CUtensorMap *map, CUtensorMapDataType dtype, size_t elem
                         uint64_t rows, uint64_t cols, uint64_t row_stride_bytes, uint32_t box_rows,
                         uint32_t box_cols, TmaSwizzle swizzle);
 
+// Raises a kernel's dynamic shared-memory limit to `bytes`; does the CUDA call once per (kernel, device).
+bool ensure_dynamic_smem(const void *kernel, size_t bytes);
+
 #ifdef __CUDACC__
 // ---------------------------------------------------------------------------------------------
 // Device
@@ -68,13 +71,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // kernel drains and exits instead of hanging the GPU.
 constexpr uint32_t kWaitLimit = 1u << 22;
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *status) {
-    for (uint32_t i = 0; i < kWaitLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, int32_t *status, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 128) __nanosleep(64);
     }
     if (status) atomicExch(status, (int32_t)DMR_ERR_TIMEOUT);
     return false;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *status) {
+    return mbar_wait_limited(bar, parity, status, kWaitLimit);
 }
 
 // The same bounded wait for a thread that has nothing to do until the phase completes and shares
