@@ -66,7 +66,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             if r.returncode != 0:
                 raise subprocess.CalledProcessError(r.returncode, f"nvcc {src}")
     objs = [_obj(s) for s in sources()]
-    subprocess.run([nvcc, "--shared", "-o", LIB] + objs, check=True)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "--shared", "-o", LIB] + objs, check=True)
     return LIB
 
 

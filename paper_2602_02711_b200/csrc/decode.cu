@@ -32,9 +32,9 @@
 //
 // Launch chains.  The kernel lets its successor start at once (programmatic dependent launch) and asks for
 // more than half of an SM's shared memory, so that an SM never holds two CTAs of these kernels: the
-// successor's CTA moves in when this kernel's CTA on that SM has finished, asks for its share of the weights
-// to be brought into the L2 (bulk prefetches consume no value), fills its rings and only then waits for its
-// predecessor.  (With two CTAs per SM the successor's CTAs land wherever a slot happens to be free - two on
+// successor's CTA moves in when this kernel's CTA on that SM has finished, fills its rings and only then waits
+// for its predecessor.  (Bulk prefetches of the CTA's whole share into the L2 were tried on top of the rings and
+// cost more issue slots than they saved: 159 against 147 us per sweep of twelve layers.)  (With two CTAs per SM the successor's CTAs land wherever a slot happens to be free - two on
 // some SMs, none on others - and the kernel runs at the pace of the doubly loaded SMs; measured with in-kernel
 // time stamps.)  Weights, scales and zero points are read before the wait: they must not be produced by a
 // kernel that releases its dependents early (the library's own kernels that write weights never do).
@@ -48,8 +48,6 @@ namespace dmr {
 
 namespace {
 
-constexpr int kPrefetchPiece = 4096;              // bytes per bulk prefetch instruction
-constexpr long long kPrefetchAhead = 192 * 1024;  // bytes of weights a CTA keeps requested ahead of its loads
 
 struct DecodeArgs {
     const uint16_t *X;        // [*][K] bf16
@@ -65,7 +63,6 @@ struct DecodeArgs {
     int g_size;
     int tiles;                // ceil(N / tile rows)
     int nchunks;              // K / chunk size
-    int pf_tiles;             // tiles whose weights are requested ahead
     int sz_stage;             // 1: a tile's scales and zero points are copied to shared memory ahead of time
     int sz_vec;               // 1: the entries of a box's groups are consecutive, aligned and read with one load each
     int sz_zoff, sz_stride;   // shared-memory offset of a tile's zero points; bytes between the tile buffers
@@ -76,12 +73,6 @@ __device__ __forceinline__ uint4 ldg_v4(const void *p) {
     asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
-// Asks the memory system to bring [p, p + bytes) into the L2; nothing is written anywhere else and
-// nothing waits for it.  p and bytes are multiples of 16.
-__device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void prefetch_l2_line(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 // Copies `bytes` (a multiple of 16, both addresses 16-byte aligned) from global to shared memory; completes on `bar`.
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src),
@@ -151,7 +142,6 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
     const int pg = (g >> 1) | ((g & 1) << 2);  // box row of fragment row g: 0, 4, 1, 5, ... (bank-conflict-free under the swizzle)
     const int t0 = (int)(((long long)blockIdx.x * a.tiles) / gridDim.x);
     const int t1 = (int)(((long long)(blockIdx.x + 1) * a.tiles) / gridDim.x);
-    const size_t row_bytes = (size_t)a.K >> 1;
     const uint32_t ring = base + (uint32_t)warp * (D * Cfg::STAGE_BYTES);
     const uint32_t bars = base + Cfg::BAR_OFF + (uint32_t)warp * (D * 8);
     const uint32_t szbars = base + Cfg::BAR_OFF + WARPS * D * 8;
@@ -170,23 +160,6 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
     }
     __syncthreads();
     pdl_launch_dependents();
-
-    // ---- requests for this CTA's weights, scales and zero points (no value is looked at) ----
-    auto prefetch_tiles = [&](int ta, int tb) {  // tiles [ta, tb)
-        const long long r0 = (long long)ta * TILE, r1 = min((long long)tb * TILE, (long long)a.N);
-        if (r1 <= r0) return;
-        const char *wb = reinterpret_cast<const char *>(a.qweight) + r0 * row_bytes;
-        const long long wbytes = (r1 - r0) * (long long)row_bytes;
-        for (long long o = (long long)threadIdx.x * kPrefetchPiece; o < wbytes; o += (long long)THREADS * kPrefetchPiece)
-            prefetch_l2_bulk(wb + o, (uint32_t)min((long long)kPrefetchPiece, wbytes - o));
-        const char *sb = reinterpret_cast<const char *>(a.scales) + r0 * a.G * 2;
-        const long long sbytes = (r1 - r0) * a.G * 2;
-        for (long long o = (long long)threadIdx.x * 128; o < sbytes; o += (long long)THREADS * 128) prefetch_l2_line(sb + o);
-        const char *zb = reinterpret_cast<const char *>(a.zeros) + r0 * a.G;
-        const long long zbytes = (r1 - r0) * a.G;
-        for (long long o = (long long)threadIdx.x * 128; o < zbytes; o += (long long)THREADS * 128) prefetch_l2_line(zb + o);
-    };
-    if (t1 > t0) prefetch_tiles(t0, min(t1, t0 + a.pf_tiles));
 
     // ---- a tile's scales and zero points into shared memory (two contiguous blocks of the tables) ----
     int sz_issued = 0;
@@ -306,7 +279,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                         }
                     }
             }
-#pragma unroll
+#pragma unroll(NT == 1 ? CPB : 1)
             for (int sub = 0; sub < CPB; ++sub) {
                 if (sub >= nsub) break;
                 const int chunk = box * CPB + sub;
@@ -426,7 +399,6 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
             }
         }
         // ---- end of a tile: add the warps' sums in warp order and write the outputs ----
-        if (tile + a.pf_tiles < t1) prefetch_tiles(tile + a.pf_tiles, tile + a.pf_tiles + 1);
         float *rbuf = red + (size_t)(Cfg::RED_BUFS == 2 ? (tl & 1) : 0) * WARPS * (NACC * 32);
 #pragma unroll
         for (int r = 0; r < R; ++r)
@@ -494,9 +466,6 @@ dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
     a.nchunks = a.K / Cfg::CHUNK_K;
     int ctas = device_sm_count();
     if (ctas > a.tiles) ctas = a.tiles;
-    const long long tile_bytes = (long long)TILE * (a.K / 2);
-    a.pf_tiles = (int)((kPrefetchAhead + tile_bytes - 1) / tile_bytes);
-    if (a.pf_tiles < 2) a.pf_tiles = 2;
     // A tile's scales and zero points are two contiguous blocks of the tables: they are copied to shared memory ahead
     // of time when every tile is whole, the blocks are 16-byte aligned and three tiles' worth stay small.
     const size_t tile_entries = (size_t)TILE * a.G;
