@@ -148,17 +148,19 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
     const uint32_t szbuf = base + Cfg::SZ_OFF;
     const int nboxes = (a.nchunks + CPB - 1) / CPB;
 
+    // Every warp sets up its own ring and starts its first copies at once; the barriers of the shared scale / zero-point
+    // buffers are warp 0's, and the one CTA-wide barrier that makes them visible comes after the copies are under way.
+    if (threadIdx.x == 0) prefetch_tensor_map(&wmap);
     if (lane == 0) {
 #pragma unroll
         for (int d = 0; d < D; ++d) mbar_init(bars + 8 * d, 1);
         if (warp == 0) {
 #pragma unroll
             for (int d = 0; d < kSzBuffers; ++d) mbar_init(szbars + 8 * d, 1);
-            prefetch_tensor_map(&wmap);
         }
         fence_barrier_init();
     }
-    __syncthreads();
+    __syncwarp();
     pdl_launch_dependents();
 
     // ---- a tile's scales and zero points into shared memory (two contiguous blocks of the tables) ----
@@ -172,11 +174,6 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
         bulk_copy_g2s(szbuf + d * a.sz_stride + a.sz_zoff, a.zeros + (size_t)tile * n_entries, n_entries, szbars + 8 * d);
         ++sz_issued;
     };
-    if (threadIdx.x == 0) {
-        issue_sz(t0);
-        issue_sz(t0 + 1);
-    }
-
     // ---- this warp's list of steps: tiles t0, t0 + 1, ...; boxes warp, warp + WARPS, ... of each ----
     const bool has_boxes = warp < nboxes;
     bool ok = true;  // false once a bounded wait ran out: the warp stops copying, waiting and storing but still meets every barrier
@@ -197,6 +194,11 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
     };
 #pragma unroll
     for (int d = 0; d < D; ++d) issue();
+    if (threadIdx.x == 0) {
+        issue_sz(t0);
+        issue_sz(t0 + 1);
+    }
+    __syncthreads();  // warp 0's barriers are set up before anyone waits on them
 
     pdl_wait();
     const int rows = a.count ? min(*a.count - a.coff, a.M) : a.M;
