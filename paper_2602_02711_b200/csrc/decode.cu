@@ -64,7 +64,7 @@ struct DecodeArgs {
     int tiles;                // ceil(N / tile rows)
     int nchunks;              // K / chunk size
     int sz_stage;             // 1: a tile's scales and zero points are copied to shared memory ahead of time
-    int sz_vec;               // 1: the entries of a box's groups are consecutive, aligned and read with one load each
+    int sz_vec;               // 1: the entries of a box's groups are consecutive, aligned and read with one load each (shared or global)
     int sz_zoff, sz_stride;   // shared-memory offset of a tile's zero points; bytes between the tile buffers
 };
 
@@ -270,14 +270,26 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const uint32_t o = szo[r][h] + (uint32_t)grp0;
-                        if constexpr (CPB == 2) {
-                            scv[r][h][0] = lds_u32(sbase + 2 * o);
-                            zpv[r][h] = lds_u16(zbase + o);
-                        } else {
-                            const uint2 v = lds_v2(sbase + 2 * o);
-                            scv[r][h][0] = v.x;
-                            scv[r][h][CPB / 2 - 1] = v.y;
-                            zpv[r][h] = lds_u32(zbase + o);
+                        if (a.sz_stage) {
+                            if constexpr (CPB == 2) {
+                                scv[r][h][0] = lds_u32(sbase + 2 * o);
+                                zpv[r][h] = lds_u16(zbase + o);
+                            } else {
+                                const uint2 v = lds_v2(sbase + 2 * o);
+                                scv[r][h][0] = v.x;
+                                scv[r][h][CPB / 2 - 1] = v.y;
+                                zpv[r][h] = lds_u32(zbase + o);
+                            }
+                        } else {  // tables too large to stage: the same aligned loads from global memory
+                            if constexpr (CPB == 2) {
+                                scv[r][h][0] = __ldg(reinterpret_cast<const uint32_t *>(a.scales + o));
+                                zpv[r][h] = __ldg(reinterpret_cast<const uint16_t *>(a.zeros + o));
+                            } else {
+                                const uint2 v = __ldg(reinterpret_cast<const uint2 *>(a.scales + o));
+                                scv[r][h][0] = v.x;
+                                scv[r][h][CPB / 2 - 1] = v.y;
+                                zpv[r][h] = __ldg(reinterpret_cast<const uint32_t *>(a.zeros + o));
+                            }
                         }
                     }
             }
@@ -476,7 +488,8 @@ dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
     a.sz_stage = (a.N % TILE == 0 && tile_entries % 16 == 0 && ((uintptr_t)a.scales % 16) == 0 && ((uintptr_t)a.zeros % 16) == 0 &&
                   (size_t)kSzBuffers * a.sz_stride <= kSzBudget) ? 1 : 0;
     // a box covers CPB consecutive groups and every row's entries start at a multiple of CPB
-    a.sz_vec = (a.sz_stage && a.g_size == Cfg::CHUNK_K && a.G % Cfg::CPB == 0) ? 1 : 0;
+    a.sz_vec = (a.g_size == Cfg::CHUNK_K && a.G % Cfg::CPB == 0 &&
+                (a.sz_stage || (((uintptr_t)a.scales % (2 * Cfg::CPB)) == 0 && ((uintptr_t)a.zeros % Cfg::CPB) == 0))) ? 1 : 0;
     const size_t smem = Cfg::SMEM + (a.sz_stage ? (size_t)kSzBuffers * a.sz_stride : 0);
     CUtensorMap wmap;
     const uint64_t rb = (uint64_t)a.K / 2;

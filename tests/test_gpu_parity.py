@@ -110,14 +110,12 @@ def run_lowbit_case(M, N, K, bits, group, seed=0, outlier=0.0):
     Y32 = dmr.dmr_lowbit_linear(Xd, q, OUT_F32)
     Y16 = dmr.dmr_lowbit_linear(Xd, q, OUT_BF16)
     Yref = oracle.lowbit_linear(X, *ref, bits=bits, group=group)
-    Yrefb = oracle.lowbit_linear(X, *ref, bits=bits, group=group, rounded=True)
     y32 = Y32.cpu().numpy().astype(np.float64)
     assert rel_err(y32, Yref) <= TOL
     # sharper check: the decode kernels and the split-K tensor-core kernel multiply exact integers
     # (only fp32 summation order differs from the oracle); the persistent prefill kernel (M > 32)
     # rounds each dequantized weight once to fp16's 11 significant bits
     assert rel_err(y32, Yref) <= (TOL_ROUNDED if M <= 32 else TOL_PREFILL)
-    del Yrefb
     # bf16 output = nearest bf16 of the same accumulators
     assert torch.equal(Y16, Y32.to(torch.bfloat16))
     # determinism
@@ -139,10 +137,10 @@ def test_config1_lowbit_linear(M):
     (16, 328, 512, 8, 128),
     (1, 24, 128, 4, 128),      # smallest K the decode kernel takes
     (2, 40, 160, 4, 32),       # K not a multiple of 128: any-shape kernel
-    (24, 1000, 1024, 4, 128),  # 17 .. 32 rows: the 32-row instance of the decode kernel
-    (32, 520, 2048, 8, 0),
-    (17, 4096, 4096, 4, 64),   # ... in cluster mode (clusters of four)
-    (31, 22016, 512, 4, 128),  # ... with more feature groups per cluster than fit at once
+    (24, 1000, 1024, 4, 128),  # 17 .. 32 rows: two chunks of the 16-row instance of the 4-bit decode kernel
+    (32, 520, 2048, 8, 0),     # 8-bit: the 32-row instance of the streaming kernel
+    (17, 4096, 4096, 4, 64),   # g = 64, one full and one one-row chunk
+    (31, 22016, 512, 4, 128),  # many tiles per CTA, two boxes per row
     (40, 300, 512, 4, 128),    # M above the decode limit: tensor-core GEMM, ragged N and M
     (33, 136, 384, 8, 0),
     (64, 256, 4096, 4, 128),   # few tiles, long K: split-K with ordered reduction
@@ -156,15 +154,15 @@ def test_lowbit_linear_shapes(M, N, K, bits, group):
 
 
 @pytest.mark.parametrize("M,N,K,bits,group", [
-    (8, 22016, 2048, 4, 128),  # 172 feature groups over at most 33 clusters: more than fit into shared memory at once (two rounds)
-    (3, 4224, 768, 4, 128),    # 3 steps per feature group: five of the eight ranks of a cluster have no k slice
-    (7, 1000, 4096, 8, 128),   # INT8, ragged N: 8 feature groups, 8 clusters
-    (1, 4096, 4096, 4, 64),    # g = 64 (two groups per 128-code unit), one feature group per cluster
-    (8, 136, 11008, 4, 0),     # per-channel scales, 43 steps per group: uneven k slices (5 and 6 steps)
+    (8, 22016, 2048, 4, 128),  # 688 tiles of 32 rows, 8 boxes per row: half of the warps have no box
+    (3, 4224, 768, 4, 128),    # 3 boxes per row: most warps idle, sums of three warps
+    (7, 1000, 4096, 8, 128),   # INT8, ragged N: streaming kernel in cluster mode (8 feature groups, 8 clusters)
+    (1, 4096, 4096, 4, 64),    # g = 64 (64-wide chunks, four per box)
+    (8, 136, 11008, 4, 0),     # per-channel scales (tables not staged as pairs), 43 boxes per row: uneven shares (2 and 3 boxes)
 ])
 def test_lowbit_linear_cluster_mode_shapes(M, N, K, bits, group):
-    """Small layers with up to 8 rows: the CTAs of a thread-block cluster split each feature group's k
-    range and add their sums through distributed shared memory."""
+    """Layers with up to 8 rows whose k range divides unevenly among the warps of a CTA (4-bit decode kernel)
+    or among the CTAs of a thread-block cluster (8-bit streaming kernel)."""
     run_lowbit_case(M, N, K, bits, group, seed=5)
 
 
@@ -295,9 +293,9 @@ def test_routed_linear_int8_and_ragged():
 
 @pytest.mark.parametrize("M,N,K", [(24, 1000, 4096), (31, 4096, 1024), (20, 22016, 512)])
 def test_routed_rows_move_between_chunks(M, N, K):
-    """17 to 32 rows run as chunks of 16: a routed call moves rows from one chunk to another, and they must
-    still come out bit for bit as in the unrouted call (every chunk uses the same kernel and summation
-    order), on layers large enough for feature groups to be shared between CTAs or clusters."""
+    """17 to 32 rows run as chunks: a routed call moves rows from one chunk to another, and they must
+    still come out bit for bit as in the unrouted call (every chunk uses the same kernel instance and summation
+    order)."""
     mask = inputs.precision_mask(M, 0.4, seed=M)
     routed_case(M, N, K, 4, 128, mask)
 
@@ -357,10 +355,10 @@ def test_lowbit_linear_host_matches_device_call():
 # ---------------- full-size shapes, sampled outputs ----------------
 
 def test_decode_launch_chains_are_repeatable():
-    """Back-to-back launches on one stream and one workspace (programmatic dependent launch lets a kernel
-    start while its predecessor drains): every repetition must give the bits of the first one, and that
-    one must match the oracle.  Mixes layers that take the contiguous split (counters and partial sums
-    in the workspace) with layers that run in clusters, and 1-, 8- and 16-row batches."""
+    """Back-to-back launches of the 4-bit decode kernel on one stream and one workspace (programmatic dependent
+    launch lets a kernel start while its predecessor drains): every repetition must give the bits of the first one,
+    and that one must match the oracle.  Layers with one to several tiles per CTA, 1-, 8- and 16-row batches.  (The
+    streaming kernel's chains, with counters and partial sums in the workspace, are in test_gpu_full_size.py.)"""
     fmt = QFormat(4, 128)
     cases = []
     for (N, K, M) in [(3000, 11008, 1), (1024, 4096, 8), (3000, 11008, 16), (640, 2048, 16), (2200, 16384, 4)]:
