@@ -103,7 +103,7 @@ def quantize(W: np.ndarray, bits: int = 4, group: int = 128, return_codes: bool 
     W = _c(W, np.uint16)
     N, K = W.shape
     g = group_of(K, group)
-    if K % g != 0 or K % (32 // bits) != 0:
+    if K % g != 0 or K % (32 if bits == 3 else 32 // bits) != 0:
         raise OracleError(ERR_ARG)
     G = K // g
     qweight = np.zeros((N, K * bits // 32), dtype=np.uint32)

@@ -28,7 +28,13 @@
  *   W  [N][K] bf16 bit patterns (uint16), N = out features, K = in features
  *   X  [M][K] bf16 bit patterns,          M = tokens / concurrent agent steps
  *   qweight [N][K*bits/32] uint32: 4-bit code k of a row sits in word k/8 at bits 4*(k%8)..+3;
- *                                  8-bit code k sits in word k/4 at bits 8*(k%4)..+7
+ *                                  8-bit code k sits in word k/4 at bits 8*(k%4)..+7;
+ *                                  3-bit codes (the W3A16 variant of Sec. 5 / App. "Quantization Detail"): every 32
+ *                                  codes take three words.  Code i of the block, i < 30, sits in word i/10 at bits
+ *                                  3*(i%10)..+2 when i%10 < 5 and at bits 16+3*(i%10-5)..+2 otherwise (five codes in
+ *                                  each half-word, bit 15 and bit 31 left over); bit b of code 30 is bit 15 of word b,
+ *                                  bit b of code 31 is bit 31 of word b.  (The paper gives no 3-bit layout: its W3
+ *                                  checkpoint is expanded to fp16 at load time.  This one is defined by this build.)
  *   scales  [N][K/g] bf16 bits,  zeros [N][K/g] uint8
  *   Y  [M][N] binary64
  */
@@ -95,39 +101,74 @@ double oracle_bf16_to_f64(uint16_t b) { return bf16_to_f64(b); }
 /* ---------- packing ---------- */
 
 static int format_ok(int K, int bits, int g) {
-    if (bits != 4 && bits != 8) return 0;
+    if (bits != 3 && bits != 4 && bits != 8) return 0;
     if (K <= 0 || g <= 0 || K % g != 0) return 0;
-    if (K % (32 / bits) != 0) return 0;
+    if (bits == 3 ? K % 32 != 0 : K % (32 / bits) != 0) return 0;
     return 1;
+}
+
+static int words_per_row(int K, int bits) { return bits == 3 ? K / 32 * 3 : K / (32 / bits); }
+
+/* where code i (0..29) of a 32-code block of 3-bit codes sits: word index and shift */
+static void w3_place(int i, int *word, int *shift) {
+    *word = i / 10;
+    int j = i % 10;
+    *shift = j < 5 ? 3 * j : 16 + 3 * (j - 5);
+}
+
+/* code k of one packed row */
+static uint32_t code_at(const uint32_t *row, int k, int bits) {
+    if (bits == 3) {
+        const uint32_t *w = row + (size_t)(k / 32) * 3;
+        int i = k % 32;
+        if (i < 30) {
+            int word, shift;
+            w3_place(i, &word, &shift);
+            return (w[word] >> shift) & 7u;
+        }
+        int bit = i == 30 ? 15 : 31;
+        return ((w[0] >> bit) & 1u) | (((w[1] >> bit) & 1u) << 1) | (((w[2] >> bit) & 1u) << 2);
+    }
+    int per = 32 / bits;
+    return (row[k / per] >> (bits * (k % per))) & ((1u << bits) - 1u);
 }
 
 /* codes [N][K] uint8 (each < 2^bits) -> qweight [N][K*bits/32] */
 int oracle_pack(const uint8_t *codes, int N, int K, int bits, uint32_t *qweight) {
-    if (bits != 4 && bits != 8) return ORACLE_ERR_ARG;
-    int per = 32 / bits;
-    if (K % per != 0) return ORACLE_ERR_ARG;
-    int words = K / per;
-    for (int n = 0; n < N; ++n)
-        for (int j = 0; j < words; ++j) {
-            uint32_t w = 0;
-            for (int i = 0; i < per; ++i)
-                w |= (uint32_t)codes[(size_t)n * K + (size_t)j * per + i] << (bits * i);
-            qweight[(size_t)n * words + j] = w;
+    if (bits != 3 && bits != 4 && bits != 8) return ORACLE_ERR_ARG;
+    if (bits == 3 ? K % 32 != 0 : K % (32 / bits) != 0) return ORACLE_ERR_ARG;
+    int words = words_per_row(K, bits);
+    for (int n = 0; n < N; ++n) {
+        uint32_t *row = qweight + (size_t)n * words;
+        for (int j = 0; j < words; ++j) row[j] = 0;
+        for (int k = 0; k < K; ++k) {
+            uint32_t c = codes[(size_t)n * K + k];
+            if (bits == 3) {
+                uint32_t *w = row + (size_t)(k / 32) * 3;
+                int i = k % 32;
+                if (i < 30) {
+                    int word, shift;
+                    w3_place(i, &word, &shift);
+                    w[word] |= (c & 7u) << shift;
+                } else {
+                    int bit = i == 30 ? 15 : 31;
+                    for (int b = 0; b < 3; ++b) w[b] |= ((c >> b) & 1u) << bit;
+                }
+            } else {
+                int per = 32 / bits;
+                row[k / per] |= (c & ((1u << bits) - 1u)) << (bits * (k % per));
+            }
         }
+    }
     return ORACLE_OK;
 }
 
 int oracle_unpack(const uint32_t *qweight, int N, int K, int bits, uint8_t *codes) {
-    if (bits != 4 && bits != 8) return ORACLE_ERR_ARG;
-    int per = 32 / bits;
-    if (K % per != 0) return ORACLE_ERR_ARG;
-    int words = K / per;
-    uint32_t maskv = (1u << bits) - 1u;
+    if (bits != 3 && bits != 4 && bits != 8) return ORACLE_ERR_ARG;
+    if (bits == 3 ? K % 32 != 0 : K % (32 / bits) != 0) return ORACLE_ERR_ARG;
+    int words = words_per_row(K, bits);
     for (int n = 0; n < N; ++n)
-        for (int k = 0; k < K; ++k) {
-            uint32_t w = qweight[(size_t)n * words + k / per];
-            codes[(size_t)n * K + k] = (uint8_t)((w >> (bits * (k % per))) & maskv);
-        }
+        for (int k = 0; k < K; ++k) codes[(size_t)n * K + k] = (uint8_t)code_at(qweight + (size_t)n * words, k, bits);
     return ORACLE_OK;
 }
 
@@ -175,7 +216,7 @@ int oracle_quantize(const uint16_t *W, int N, int K, int bits, int group,
                     uint32_t *qweight, uint16_t *scales, uint8_t *zeros, uint8_t *codes_out) {
     int g = group == 0 ? K : group;
     if (N <= 0 || !format_ok(K, bits, g)) return ORACLE_ERR_ARG;
-    int G = K / g, words = K / (32 / bits);
+    int G = K / g, words = words_per_row(K, bits);
     int err = ORACLE_OK;
 #pragma omp parallel for schedule(static)
     for (int n = 0; n < N; ++n) {
@@ -204,12 +245,11 @@ int oracle_dequantize(const uint32_t *qweight, const uint16_t *scales, const uin
                       int N, int K, int bits, int group, double *What, uint16_t *What_bf16) {
     int g = group == 0 ? K : group;
     if (N <= 0 || !format_ok(K, bits, g)) return ORACLE_ERR_ARG;
-    int G = K / g, per = 32 / bits, words = K / per;
-    uint32_t maskv = (1u << bits) - 1u;
+    int G = K / g, words = words_per_row(K, bits);
 #pragma omp parallel for schedule(static)
     for (int n = 0; n < N; ++n)
         for (int k = 0; k < K; ++k) {
-            uint32_t q = (qweight[(size_t)n * words + k / per] >> (bits * (k % per))) & maskv;
+            uint32_t q = code_at(qweight + (size_t)n * words, k, bits);
             double s = bf16_to_f64(scales[(size_t)n * G + k / g]);
             double z = (double)zeros[(size_t)n * G + k / g];
             double v = s * ((double)q - z);
@@ -224,9 +264,8 @@ int oracle_dequantize(const uint32_t *qweight, const uint16_t *scales, const uin
 /* one dequantized weight; rounded != 0 gives the nearest-bf16 version (diagnostic) */
 static double dq_weight(const uint32_t *qweight, const uint16_t *scales, const uint8_t *zeros,
                         int K, int bits, int g, int n, int k, int rounded) {
-    int G = K / g, per = 32 / bits, words = K / per;
-    uint32_t maskv = (1u << bits) - 1u;
-    uint32_t q = (qweight[(size_t)n * words + k / per] >> (bits * (k % per))) & maskv;
+    int G = K / g, words = words_per_row(K, bits);
+    uint32_t q = code_at(qweight + (size_t)n * words, k, bits);
     double s = bf16_to_f64(scales[(size_t)n * G + k / g]);
     double z = (double)zeros[(size_t)n * G + k / g];
     double v = s * ((double)q - z);
