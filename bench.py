@@ -239,7 +239,7 @@ def run_ours(args):
     peaks = load_peaks()
     fmt = QFormat(BITS, GROUP)
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost", "kl", "crossover"}
+    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost", "w3", "kl", "crossover"}
 
     def bf16_dev(bits_np):
         return torch.from_numpy(bits_np.view(np.int16)).view(torch.bfloat16).to(dev)
@@ -560,6 +560,49 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, l2_b
         out["layer_cost_7b"] = {k: {"t_high_us": round(v["t_high_us_per_layer"], 1), "t_low_us": round(v["t_low_us_per_layer"], 1),
                                     "ratio": round(v["t_high_over_t_low"], 2)} for k, v in lc.items()}
 
+    if "w3" in sections:
+        # The 3-bit variant (W3A16 g=128, Sec. 5 / App. "Quantization Detail") against the 4-bit one on the same 7B-class
+        # layer: per-token decode time of the four linears chained in one CUDA graph, weights rotated over copies larger
+        # than the L2.  The paper has no 3-bit kernel and projects T_W3 = T_W4 / 1.15 (App. "Latency calibration");
+        # this is the measured ratio for this library's kernels.
+        w3 = {}
+        f3, f4 = QF(3, 128), QF(4, 128)
+        layer_w4 = sum(N * K // 2 for N, K in inputs.LAYER_7B.values())
+        layer_w3 = sum(N * K * 3 // 8 for N, K in inputs.LAYER_7B.values())
+        ncopy = copies_beyond_l2(layer_w3, l2_bytes)
+        Q3s, Q4s = [], []
+        for c in range(ncopy):
+            l3, l4 = {}, {}
+            for i, (n, (N, K)) in enumerate(inputs.LAYER_7B.items()):
+                W = randw(N, K, 171 + 7 * c + i)
+                l3[n] = dmr.dmr_quantize(W, f3)
+                l4[n] = dmr.dmr_quantize(W, f4)
+                del W
+            Q3s.append(l3)
+            Q4s.append(l4)
+        for M in (1, 8, 16):
+            Xs = {n: randx(M, K, 3) for n, (N, K) in inputs.LAYER_7B.items()}
+            Ys = {n: torch.empty((M, N), dtype=torch.bfloat16, device=dev) for n, (N, K) in inputs.LAYER_7B.items()}
+            ws3 = dmr.new_workspace(0, M, 22016, 11008, f3, dev)
+            ws4 = dmr.new_workspace(0, M, 22016, 11008, f4, dev)
+
+            def layer_call(Qs, ws):
+                def call(c):
+                    for n in inputs.LAYER_7B:
+                        dmr.dmr_lowbit_linear(Xs[n], Qs[c][n], OUT_BF16, Y=Ys[n], workspace=ws)
+                return call
+
+            t4 = time_rotating(layer_call(Q4s, ws4), ncopy, reps=60)
+            t3 = time_rotating(layer_call(Q3s, ws3), ncopy, reps=60)
+            w3[f"M{M}"] = {"t_w4_us_per_layer": t4 * 1e6, "t_w3_us_per_layer": t3 * 1e6, "t_w4_over_t_w3": t4 / t3,
+                           "w4_weight_gbs": layer_w4 / t4 / 1e9, "w3_weight_gbs": layer_w3 / t3 / 1e9,
+                           "w3_frac_hbm": layer_w3 / t3 / 1e9 / peaks["hbm_gbs"],
+                           "paper_projection_t_w4_over_t_w3": 1.15}
+        del Q3s, Q4s
+        emit_section("w3_vs_w4_decode_7b", w3)
+        out["w3_vs_w4_decode_7b"] = {k: {"t_w4_us": round(v["t_w4_us_per_layer"], 1), "t_w3_us": round(v["t_w3_us_per_layer"], 1),
+                                         "ratio": round(v["t_w4_over_t_w3"], 3)} for k, v in w3.items()}
+
     if "crossover" in sections:
         # 32B-class gate and down linears, INT4 g=64 and INT8 per-channel, M = 1 .. 256, 1 % outlier channels x20,
         # with the library's default dispatch (decode kernels up to 32 rows, tensor-core kernels above): where
@@ -630,7 +673,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost,kl (default: all; none = headline only)")
+    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost,w3,kl (default: all; none = headline only)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

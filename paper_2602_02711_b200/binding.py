@@ -27,7 +27,7 @@ class DmrError(RuntimeError):
 
 
 class QFormat(ctypes.Structure):
-    """dmr_qformat_t: bits in {4, 8}; group_size 0 = one group per output row."""
+    """dmr_qformat_t: bits in {3, 4, 8}; group_size 0 = one group per output row."""
     _fields_ = [("bits", ctypes.c_int32), ("group_size", ctypes.c_int32)]
 
     def group(self, K: int) -> int:

@@ -152,7 +152,8 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
         }
         return launch_gemm(Xin, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.partial, ws.status, st);
     }
-    if (f.bits == 4 && decode_w4_enabled() && decode_w4_supported(M < kDecodeChunk ? M : kDecodeChunk, N, K, g)) {
+    const bool dec3 = f.bits == 3 && decode_w3_supported(M < kDecodeChunk ? M : kDecodeChunk, N, K, g);
+    if (dec3 || (f.bits == 4 && decode_w4_enabled() && decode_w4_supported(M < kDecodeChunk ? M : kDecodeChunk, N, K, g))) {
         // chunks of up to 16 rows; the kernel gathers the rows of a routed call itself
         for (int m0 = 0; m0 < M; m0 += kDecodeChunk) {
             const int mc = M - m0 < kDecodeChunk ? M - m0 : kDecodeChunk;
@@ -166,7 +167,8 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
                 Xc = X + (size_t)m0 * K;
                 Yc = reinterpret_cast<char *>(Y) + (size_t)m0 * N * ysz;
             }
-            dmr_status_t r = launch_decode_w4(Xc, mc, s, qweight, scales, zeros, N, K, g, Yc, out, ws.status, st, M);
+            dmr_status_t r = dec3 ? launch_decode_w3(Xc, mc, s, qweight, scales, zeros, N, K, g, Yc, out, ws.status, st, M)
+                                  : launch_decode_w4(Xc, mc, s, qweight, scales, zeros, N, K, g, Yc, out, ws.status, st, M);
             if (r != DMR_OK) return r;
         }
         return DMR_OK;
@@ -292,7 +294,7 @@ size_t dmr_workspace_bytes(dmr_op_t op, int M, int N, int K, dmr_qformat_t f) {
 dmr_status_t dmr_quantize(const void *W_bf16, int N, int K, dmr_qformat_t f, void *qweight, void *scales,
                           void *zeros, int32_t *dev_status, void *stream) {
     if (N < 1 || K < 1 || !W_bf16 || !qweight || !scales || !zeros) return DMR_ERR_INVALID_ARG;
-    if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
+    if (f.bits != 3 && f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
     if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
     if (!aligned16(W_bf16) || !aligned16(qweight)) return DMR_ERR_ALIGNMENT;
     return launch_quantize(reinterpret_cast<const uint16_t *>(W_bf16), N, K, f.bits, group_of(K, f),
@@ -304,7 +306,7 @@ dmr_status_t dmr_dequantize(const void *qweight, const void *scales, const void 
                             dmr_qformat_t f, void *W_out, dmr_out_t out, void *stream) {
     if (N < 1 || K < 1 || !qweight || !scales || !zeros || !W_out) return DMR_ERR_INVALID_ARG;
     if (out != DMR_OUT_BF16 && out != DMR_OUT_F32) return DMR_ERR_INVALID_ARG;
-    if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
+    if (f.bits != 3 && f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
     if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
     if (!aligned16(qweight) || !aligned16(W_out)) return DMR_ERR_ALIGNMENT;
     return launch_dequantize(reinterpret_cast<const uint32_t *>(qweight), reinterpret_cast<const uint16_t *>(scales),
@@ -318,7 +320,7 @@ dmr_status_t dmr_lowbit_linear(const void *X_bf16, int M, const void *qweight, c
     dmr_status_t r = common_checks(X_bf16, M, N, K, Y, out);
     if (r != DMR_OK) return r;
     if (!qweight || !scales || !zeros) return DMR_ERR_INVALID_ARG;
-    if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
+    if (f.bits != 3 && f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
     if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
     if (!aligned16(qweight)) return DMR_ERR_ALIGNMENT;
     if (M == 0) return DMR_OK;  // nothing to do, no workspace needed
@@ -362,7 +364,7 @@ dmr_status_t dmr_routed_linear(const void *X_bf16, int M, const uint8_t *mask, c
     if (r != DMR_OK) return r;
     if (!W_bf16 || !qweight || !scales || !zeros) return DMR_ERR_INVALID_ARG;
     if (M > 0 && !mask) return DMR_ERR_INVALID_ARG;
-    if (f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
+    if (f.bits != 3 && f.bits != 4 && f.bits != 8) return DMR_ERR_UNSUPPORTED;
     if (!format_ok(K, f)) return DMR_ERR_INVALID_ARG;
     if (!aligned16(W_bf16) || !aligned16(qweight)) return DMR_ERR_ALIGNMENT;
     if (M == 0) return DMR_OK;  // nothing to do, no workspace needed
@@ -477,6 +479,11 @@ int dmr_describe_dispatch(dmr_op_t op, int M, int N, int K, dmr_qformat_t f, cha
         }
         const GemmPlan p = gemm_plan(M, N, K, bits);
         return snprintf(buf, buf_bytes, "gemm bits=%d bn=%d splits=%d", bits, p.bn, p.splits);
+    }
+    if (!dense && bits == 3 && decode_w3_supported(M < kDecodeChunk ? M : kDecodeChunk, N, K, g)) {
+        int nt, r, warps;
+        decode_w3_plan(M, &nt, &r, &warps);
+        return snprintf(buf, buf_bytes, "decode_w3 rows=%d tile=%d warps=%d chunks=%d", 8 * nt, 16 * r, warps, (M + kDecodeChunk - 1) / kDecodeChunk);
     }
     if (!dense && bits == 4 && decode_w4_enabled() && decode_w4_supported(M < kDecodeChunk ? M : kDecodeChunk, N, K, g)) {
         int nt, r, warps;

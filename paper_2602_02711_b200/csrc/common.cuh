@@ -29,9 +29,9 @@ inline bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 
 inline int group_of(int K, dmr_qformat_t f) { return f.group_size == 0 ? K : f.group_size; }
 
-// A format is usable when: bits in {4,8}; K, g multiples of 32; g divides K.
+// A format is usable when: bits in {3,4,8}; K, g multiples of 32; g divides K.
 inline bool format_ok(int K, dmr_qformat_t f) {
-    if (f.bits != 4 && f.bits != 8) return false;
+    if (f.bits != 3 && f.bits != 4 && f.bits != 8) return false;
     if (K <= 0 || K % 32 != 0) return false;
     int g = group_of(K, f);
     if (g <= 0 || g % 32 != 0 || K % g != 0) return false;
@@ -88,8 +88,15 @@ dmr_status_t launch_decode_w4(const uint16_t *X, int M, RowSel sel, const uint32
                               const uint8_t *zeros, int N, int K, int g, void *Y, dmr_out_t out, int32_t *status,
                               cudaStream_t st, int batch_rows = 0);
 
+// The same kernel for 3-bit codes (32 codes in three words): groups and K multiples of 128.
+bool decode_w3_supported(int M, int N, int K, int g);
+dmr_status_t launch_decode_w3(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales,
+                              const uint8_t *zeros, int N, int K, int g, void *Y, dmr_out_t out, int32_t *status,
+                              cudaStream_t st, int batch_rows = 0);
+
 // What the launchers would choose for a call (for dmr_describe_dispatch).
 void decode_w4_plan(int M, int g, int *nt, int *r, int *warps);
+void decode_w3_plan(int M, int *nt, int *r, int *warps);
 void stream_plan(int M, int N, int K, int bits, int *tiles, long long *steps, int *cluster);
 void prefill_plan(int M, int N, int *bn, long long *tiles, int *ctas);
 

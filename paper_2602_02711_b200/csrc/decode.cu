@@ -53,7 +53,7 @@ struct DecodeArgs {
     const uint16_t *X;        // [*][K] bf16
     const int32_t *idx;       // routed: row of X / Y for batch slot s (nullptr = identity)
     const int32_t *count;     // routed: valid slots in the whole list (nullptr = M)
-    const uint32_t *qweight;  // [N][K / 8]
+    const uint32_t *qweight;  // [N][K bits / 32]
     const uint16_t *scales;   // [N][G] bf16
     const uint8_t *zeros;     // [N][G]
     void *Y;                  // [*][N]
@@ -108,13 +108,14 @@ __device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
 constexpr size_t kMinSmem = 116 * 1024;  // more than half of the 228 KB of an SM
 constexpr int kSzBuffers = 3;  // tiles whose scales and zero points are in shared memory at a time
 
-template <int NT, int R, int WPL, int WARPS, int D>
+template <int BITS, int NT, int R, int WPL, int WARPS, int D>
 struct DecodeCfg {
+    static_assert(BITS == 4 || (BITS == 3 && WPL == 4), "3-bit codes come in blocks of 32: chunks of 128 input features");
     static constexpr int THREADS = WARPS * 32;
     static constexpr int TILE = 16 * R;
     static constexpr int CHUNK_K = 32 * WPL;
-    static constexpr int CHUNK_BYTES = CHUNK_K / 2;
-    static constexpr int BOX_BYTES = 128;                     // bytes of a row in one TMA box (the 128-byte swizzle span)
+    static constexpr int CHUNK_BYTES = CHUNK_K * BITS / 8;
+    static constexpr int BOX_BYTES = BITS == 3 ? 96 : 128;    // bytes of a row in one TMA box (4 bits: the 128-byte swizzle span)
     static constexpr int CPB = BOX_BYTES / CHUNK_BYTES;       // chunks per box
     static constexpr int STAGE_BYTES = TILE * BOX_BYTES;
     static constexpr int NACC = R * NT * 4;
@@ -129,9 +130,9 @@ struct DecodeCfg {
 // NT: 8-row activation blocks (1 or 2).  R: 16-row weight blocks per tile.  WPL: code words per lane and
 // row in one chunk (4: chunks of 128 input features, for groups that are multiples of 128; 2: chunks of
 // 64, for groups of 64).  WARPS: warps per CTA.  D: stages of a warp's ring.
-template <int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
+template <int BITS, int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
 __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_constant__ CUtensorMap wmap, const DecodeArgs a) {
-    using Cfg = DecodeCfg<NT, R, WPL, WARPS, D>;
+    using Cfg = DecodeCfg<BITS, NT, R, WPL, WARPS, D>;
     constexpr int TILE = Cfg::TILE, CHUNK_K = Cfg::CHUNK_K, NACC = Cfg::NACC, THREADS = Cfg::THREADS, CPB = Cfg::CPB;
     extern __shared__ uint8_t smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -139,7 +140,8 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
-    const int pg = (g >> 1) | ((g & 1) << 2);  // box row of fragment row g: 0, 4, 1, 5, ... (bank-conflict-free under the swizzle)
+    // box row of fragment row g: 0, 4, 1, 5, ... for 4-bit codes (bank-conflict-free under the swizzle); 3-bit boxes are not swizzled
+    const int pg = BITS == 3 ? g : ((g >> 1) | ((g & 1) << 2));
     const int t0 = (int)(((long long)blockIdx.x * a.tiles) / gridDim.x);
     const int t1 = (int)(((long long)(blockIdx.x + 1) * a.tiles) / gridDim.x);
     const uint32_t ring = base + (uint32_t)warp * (D * Cfg::STAGE_BYTES);
@@ -324,6 +326,80 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                             }
                         }
                 }
+                float gs[R][NT][4], sx[NT][4];
+                if constexpr (BITS == 3) {
+                    // Lane (g, t) takes block t of the chunk (32 codes in three words) for rows g and g + 8 of each 16-row
+                    // block, and the 32 activations they meet.
+                    uint32_t w3[R][2][3];
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t addr = stage + (uint32_t)((r * 16 + h * 8 + g) * Cfg::BOX_BYTES + sub * Cfg::CHUNK_BYTES + t * 12);
+                            w3[r][h][0] = lds_u32(addr);
+                            w3[r][h][1] = lds_u32(addr + 4);
+                            w3[r][h][2] = lds_u32(addr + 8);
+                        }
+                    // Pair p = 5 j + i (j < 3, i < 5) is codes 10 j + i and 10 j + 5 + i of the block - the low and the high
+                    // half-word of word j at bit 3 i; pair 15 is codes 30 and 31.  Eight MMAs of two pairs each; the
+                    // one with the left-over pair goes first, so that every word of the stage has been used early.
+#pragma unroll
+                    for (int mi = 0; mi < 8; ++mi) {
+                        const int m = (mi + 7) & 7;
+                        uint32_t b[NT][2];
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+                            for (int q = 0; q < 2; ++q) {
+                                const int p = 2 * m + q;
+                                if (p == 15) {
+                                    b[nt][q] = x[nt][3][3];
+                                } else {
+                                    const int lo = 10 * (p / 5) + p % 5, hi = lo + 5;  // activations 2 v, 2 v + 1 are in word v
+                                    b[nt][q] = prmt(x[nt][lo >> 3][(lo >> 1) & 3], x[nt][hi >> 3][(hi >> 1) & 3],
+                                                    ((hi & 1) ? 0x7600u : 0x5400u) | ((lo & 1) ? 0x32u : 0x10u));
+                                }
+                            }
+                            if (mi == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                            else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                        }
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            uint32_t av[4];  // a0..a3: 128 + code, exact in bf16
+#pragma unroll
+                            for (int q = 0; q < 2; ++q)
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const int p = 2 * m + q;
+                                    uint32_t v;
+                                    if (p == 15) {
+                                        v = lop3_and_or(w3[r][h][0] >> 15, 0x00010001u, 0x43004300u);
+                                        v = lop3_and_or(w3[r][h][1] >> 14, 0x00020002u, v);
+                                        v = lop3_and_or(w3[r][h][2] >> 13, 0x00040004u, v);
+                                    } else {
+                                        const uint32_t u = w3[r][h][p / 5];
+                                        const int i = p % 5;
+                                        if (i == 0) v = lop3_and_or(u, 0x00070007u, 0x43004300u);
+                                        else if (i == 2) v = lop3_and_or(u >> 6, 0x00070007u, 0x43004300u);
+                                        else if (i == 4) v = lop3_and_or(u >> 12, 0x00070007u, 0x43004300u);
+                                        else  // bits 3..5: 128 + 8 q as it stands; (128 + 8 q) / 8 + 112 = 128 + q on the FMA pipe, exact
+                                            v = bf16x2_fma(lop3_and_or(i == 1 ? u : (u >> 6), 0x00380038u, 0x43004300u), 0x3E003E00u, 0x42E042E0u);
+                                    }
+                                    av[2 * q + h] = v;
+                                }
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                if (mi == 0) mma_bf16_16816_zero(gs[r][nt], av[0], av[1], av[2], av[3], b[nt][0], b[nt][1]);
+                                else mma_bf16_16816(gs[r][nt], av[0], av[1], av[2], av[3], b[nt][0], b[nt][1]);
+                            }
+                        }
+                        if (mi == 0 && sub == nsub - 1) {
+                            // every word of the box's last chunk has been used: request the box D ahead into the stage
+                            __syncwarp();
+                            issue();
+                        }
+                    }
+                } else {
                 uint32_t w[R][2][WPL];
 #pragma unroll
                 for (int r = 0; r < R; ++r)
@@ -342,7 +418,6 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                             w[r][h][1] = v.y;
                         }
                     }
-                float gs[R][NT][4], sx[NT][4];
 #pragma unroll
                 for (int j = 0; j < WPL; ++j) {
                     // activations paired like the codes: (x0, x4), (x1, x5) and (x2, x6), (x3, x7)
@@ -384,6 +459,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                         issue();
                     }
                 }
+                }  // 4-bit codes
                 // the next chunk's activations
                 {
                     int nc = chunk + 1;
@@ -434,7 +510,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
             const int c = e & 3, nt = (e >> 2) % NT, r = (e >> 2) / NT;
             const int slot = nt * 8 + 2 * (l & 3) + (c & 1);
             const int lg = l >> 2;
-            const int n = tile * TILE + r * 16 + ((lg >> 1) | ((lg & 1) << 2)) + 8 * (c >> 1);
+            const int n = tile * TILE + r * 16 + (BITS == 3 ? lg : ((lg >> 1) | ((lg & 1) << 2))) + 8 * (c >> 1);
             if (ok && slot < rows && n < a.N) {
                 const int row = a.idx ? a.idx[slot] : slot;
                 if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
@@ -466,14 +542,14 @@ bool decode_pdl_enabled() {
     return v != 0;
 }
 
-template <int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
+template <int BITS, int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
 dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
-    using Cfg = DecodeCfg<NT, R, WPL, WARPS, D>;
+    using Cfg = DecodeCfg<BITS, NT, R, WPL, WARPS, D>;
     constexpr int TILE = Cfg::TILE;
     // shared memory left for the copies of the scale / zero-point tables (227 KB per CTA at most)
     constexpr size_t kSzBudget = 227 * 1024 - Cfg::SMEM < 36 * 1024 ? 227 * 1024 - Cfg::SMEM : 36 * 1024;
     static_assert(Cfg::SMEM <= 227 * 1024, "ring and reduction buffers exceed an SM's shared memory");
-    auto kernel = decode_w4_kernel<NT, R, WPL, WARPS, D, OUT_F32>;
+    auto kernel = decode_w4_kernel<BITS, NT, R, WPL, WARPS, D, OUT_F32>;
     if (!ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), Cfg::SMEM + kSzBudget < kMinSmem ? kMinSmem : Cfg::SMEM + kSzBudget))
         return DMR_ERR_CUDA;
     a.tiles = (a.N + TILE - 1) / TILE;
@@ -492,9 +568,9 @@ dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
                 (a.sz_stage || (((uintptr_t)a.scales % (2 * Cfg::CPB)) == 0 && ((uintptr_t)a.zeros % Cfg::CPB) == 0))) ? 1 : 0;
     const size_t smem = Cfg::SMEM + (a.sz_stage ? (size_t)kSzBuffers * a.sz_stride : 0);
     CUtensorMap wmap;
-    const uint64_t rb = (uint64_t)a.K / 2;
+    const uint64_t rb = (uint64_t)a.K * BITS / 8;
     if (!make_tensor_map_2d(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.qweight, (uint64_t)a.N, rb, rb, TILE, Cfg::BOX_BYTES,
-                            TmaSwizzle::k128B))
+                            BITS == 3 ? TmaSwizzle::kNone : TmaSwizzle::k128B))
         return DMR_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas, 1, 1);
@@ -529,6 +605,13 @@ bool decode_w4_supported(int M, int N, int K, int g) {
     return g % 128 == 0 && K % 128 == 0;
 }
 
+// 3-bit codes: blocks of 32 codes never straddle a chunk of 128 input features, and a chunk lies inside one group.
+bool decode_w3_supported(int M, int N, int K, int g) {
+    (void)N;
+    if (M < 1 || M > 16) return false;
+    return g % 128 == 0 && K % 128 == 0;
+}
+
 // Instances as <NT, R, WPL, WARPS, D>.
 #ifndef DMR_DECODE_CFG8
 #define DMR_DECODE_CFG8 1, 2, 4, 16, 2
@@ -542,6 +625,12 @@ bool decode_w4_supported(int M, int N, int K, int g) {
 #ifndef DMR_DECODE_CFG16_G64
 #define DMR_DECODE_CFG16_G64 2, 2, 2, 8, 2
 #endif
+#ifndef DMR_DECODE3_CFG8
+#define DMR_DECODE3_CFG8 1, 2, 4, 16, 2
+#endif
+#ifndef DMR_DECODE3_CFG16
+#define DMR_DECODE3_CFG16 2, 2, 4, 8, 2
+#endif
 
 void decode_w4_plan(int M, int g, int *nt, int *r, int *warps) {
     const int cfg8[5] = {DMR_DECODE_CFG8}, cfg8g[5] = {DMR_DECODE_CFG8_G64}, cfg16[5] = {DMR_DECODE_CFG16}, cfg16g[5] = {DMR_DECODE_CFG16_G64};
@@ -551,9 +640,18 @@ void decode_w4_plan(int M, int g, int *nt, int *r, int *warps) {
     *warps = c[3];
 }
 
-dmr_status_t launch_decode_w4(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales,
-                              const uint8_t *zeros, int N, int K, int g, void *Y, dmr_out_t out, int32_t *status,
-                              cudaStream_t st, int batch_rows) {
+void decode_w3_plan(int M, int *nt, int *r, int *warps) {
+    const int cfg8[5] = {DMR_DECODE3_CFG8}, cfg16[5] = {DMR_DECODE3_CFG16};
+    const int *c = M <= 8 ? cfg8 : cfg16;
+    *nt = c[0];
+    *r = c[1];
+    *warps = c[3];
+}
+
+namespace {
+
+DecodeArgs decode_args(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales, const uint8_t *zeros,
+                       int N, int K, int g, void *Y, int32_t *status) {
     DecodeArgs a = {};
     a.X = X;
     a.idx = sel.idx;
@@ -572,14 +670,33 @@ dmr_status_t launch_decode_w4(const uint16_t *X, int M, RowSel sel, const uint32
     a.g_shift = -1;
     for (int sh = 0; sh < 31; ++sh)
         if ((1 << sh) == g) a.g_shift = sh;
+    return a;
+}
+
+}  // namespace
+
+dmr_status_t launch_decode_w4(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales,
+                              const uint8_t *zeros, int N, int K, int g, void *Y, dmr_out_t out, int32_t *status,
+                              cudaStream_t st, int batch_rows) {
+    const DecodeArgs a = decode_args(X, M, sel, qweight, scales, zeros, N, K, g, Y, status);
     const int call_rows = batch_rows > M ? batch_rows : M;
     const bool f32 = out == DMR_OUT_F32;
     if (call_rows <= 8) {
-        if (g == 64) return f32 ? launch_decode_t<DMR_DECODE_CFG8_G64, true>(a, st) : launch_decode_t<DMR_DECODE_CFG8_G64, false>(a, st);
-        return f32 ? launch_decode_t<DMR_DECODE_CFG8, true>(a, st) : launch_decode_t<DMR_DECODE_CFG8, false>(a, st);
+        if (g == 64) return f32 ? launch_decode_t<4, DMR_DECODE_CFG8_G64, true>(a, st) : launch_decode_t<4, DMR_DECODE_CFG8_G64, false>(a, st);
+        return f32 ? launch_decode_t<4, DMR_DECODE_CFG8, true>(a, st) : launch_decode_t<4, DMR_DECODE_CFG8, false>(a, st);
     }
-    if (g == 64) return f32 ? launch_decode_t<DMR_DECODE_CFG16_G64, true>(a, st) : launch_decode_t<DMR_DECODE_CFG16_G64, false>(a, st);
-    return f32 ? launch_decode_t<DMR_DECODE_CFG16, true>(a, st) : launch_decode_t<DMR_DECODE_CFG16, false>(a, st);
+    if (g == 64) return f32 ? launch_decode_t<4, DMR_DECODE_CFG16_G64, true>(a, st) : launch_decode_t<4, DMR_DECODE_CFG16_G64, false>(a, st);
+    return f32 ? launch_decode_t<4, DMR_DECODE_CFG16, true>(a, st) : launch_decode_t<4, DMR_DECODE_CFG16, false>(a, st);
+}
+
+dmr_status_t launch_decode_w3(const uint16_t *X, int M, RowSel sel, const uint32_t *qweight, const uint16_t *scales,
+                              const uint8_t *zeros, int N, int K, int g, void *Y, dmr_out_t out, int32_t *status,
+                              cudaStream_t st, int batch_rows) {
+    const DecodeArgs a = decode_args(X, M, sel, qweight, scales, zeros, N, K, g, Y, status);
+    const int call_rows = batch_rows > M ? batch_rows : M;
+    const bool f32 = out == DMR_OUT_F32;
+    if (call_rows <= 8) return f32 ? launch_decode_t<3, DMR_DECODE3_CFG8, true>(a, st) : launch_decode_t<3, DMR_DECODE3_CFG8, false>(a, st);
+    return f32 ? launch_decode_t<3, DMR_DECODE3_CFG16, true>(a, st) : launch_decode_t<3, DMR_DECODE3_CFG16, false>(a, st);
 }
 
 }  // namespace dmr

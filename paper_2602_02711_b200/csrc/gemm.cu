@@ -370,6 +370,7 @@ dmr_status_t launch_gemm_bn(int BN, const CUtensorMap &map_w, const CUtensorMap 
 bool gemm_supported(int M, int N, int K, int bits /*0 = dense*/, int g) {
     (void)N;
     if (M <= 16 || K % BK != 0) return false;
+    if (bits != 0 && bits != 4 && bits != 8) return false;
     if (bits != 0 && (g % BK != 0)) return false;
     return true;
 }

@@ -1,4 +1,4 @@
-// Weight packer: bf16 weights -> packed unsigned codes + per-group bf16 scale and u8 zero point,
+// Weight packer: bf16 weights -> packed unsigned codes (3, 4 or 8 bits) + per-group bf16 scale and u8 zero point,
 // and the matching dequantizer (test utility).
 //
 // The low-precision model is weight-only quantization of the decoder Linear layers with 16-bit
@@ -87,31 +87,71 @@ __global__ void __launch_bounds__(256) quantize_kernel(const uint16_t *__restric
             zeros[(size_t)n * G + j] = (uint8_t)z;
         }
 
-        // pass 2: codes, 8 per lane per step, packed little-endian in k
-        for (int c = lane; c < chunks; c += 32) {
-            uint4 v = *reinterpret_cast<const uint4 *>(wg + c * 8);
-            uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        // pass 2: codes, 8 per lane per step, packed little-endian in k (every lane takes every step of the loop:
+        // the 3-bit words are put together from four neighbouring lanes)
+        for (int c0 = 0; c0 < chunks; c0 += 32) {
+            const int c = c0 + lane;
+            const bool active = c < chunks;
             uint32_t q[8];
+            if (active) {
+                uint4 v = *reinterpret_cast<const uint4 *>(wg + c * 8);
+                uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < 4; ++i) {
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    double x = (double)bf16_bits_to_float(h ? (w[i] >> 16) : (w[i] & 0xFFFFu));
-                    double c2 = __dadd_rn(rint(__ddiv_rn(x, s)), z);
-                    c2 = fmin(fmax(c2, 0.0), qmax);
-                    q[2 * i + h] = (uint32_t)c2;
+                    for (int h = 0; h < 2; ++h) {
+                        double x = (double)bf16_bits_to_float(h ? (w[i] >> 16) : (w[i] & 0xFFFFu));
+                        double c2 = __dadd_rn(rint(__ddiv_rn(x, s)), z);
+                        c2 = fmin(fmax(c2, 0.0), qmax);
+                        q[2 * i + h] = (uint32_t)c2;
+                    }
                 }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) q[i] = 0;
             }
             const size_t k0 = (size_t)j * g + (size_t)c * 8;
             if (BITS == 4) {
                 uint32_t word = 0;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) word |= q[i] << (4 * i);
-                qweight[(size_t)n * (K / 8) + k0 / 8] = word;
-            } else {
+                if (active) qweight[(size_t)n * (K / 8) + k0 / 8] = word;
+            } else if (BITS == 8) {
                 uint32_t w0 = q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24);
                 uint32_t w1 = q[4] | (q[5] << 8) | (q[6] << 16) | (q[7] << 24);
-                *reinterpret_cast<uint2 *>(qweight + (size_t)n * (K / 4) + k0 / 4) = make_uint2(w0, w1);
+                if (active) *reinterpret_cast<uint2 *>(qweight + (size_t)n * (K / 4) + k0 / 4) = make_uint2(w0, w1);
+            } else {
+                // 32 codes in three words: code i < 30 in word i / 10, five codes in each half-word; the bits of codes
+                // 30 and 31 in bit 15 and bit 31 of the three words.  Four lanes hold one block of 32 codes.
+                uint32_t p[3] = {0u, 0u, 0u};
+                const int pos = (c & 3) * 8;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int i = pos + e;
+                    if (i < 30) {
+                        const int jj = i % 10;
+                        const uint32_t v = q[e] << (jj < 5 ? 3 * jj : 16 + 3 * (jj - 5));
+                        const int word = i / 10;
+                        p[0] |= word == 0 ? v : 0u;
+                        p[1] |= word == 1 ? v : 0u;
+                        p[2] |= word == 2 ? v : 0u;
+                    } else {
+                        const int bit = i == 30 ? 15 : 31;
+#pragma unroll
+                        for (int b = 0; b < 3; ++b) p[b] |= ((q[e] >> b) & 1u) << bit;
+                    }
+                }
+#pragma unroll
+                for (int b = 0; b < 3; ++b) {
+                    p[b] |= __shfl_xor_sync(0xFFFFFFFFu, p[b], 1);
+                    p[b] |= __shfl_xor_sync(0xFFFFFFFFu, p[b], 2);
+                }
+                if (active && (c & 3) == 0) {
+                    uint32_t *dst = qweight + (size_t)n * (K / 32 * 3) + k0 / 32 * 3;
+                    dst[0] = p[0];
+                    dst[1] = p[1];
+                    dst[2] = p[2];
+                }
             }
         }
     }
@@ -132,7 +172,22 @@ __global__ void __launch_bounds__(256) dequantize_kernel(const uint32_t *__restr
         const float s = bf16_bits_to_float(scales[(size_t)n * G + k0 / g]);
         const float z = (float)zeros[(size_t)n * G + k0 / g];
         uint32_t q[8];
-        if (BITS == 4) {
+        if (BITS == 3) {
+            const uint32_t *w = qweight + (size_t)n * (K / 32 * 3) + (size_t)(k0 / 32) * 3;
+            const uint32_t w0 = w[0], w1 = w[1], w2 = w[2];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = k0 % 32 + j;
+                if (i < 30) {
+                    const int jj = i % 10;
+                    const uint32_t word = i < 10 ? w0 : (i < 20 ? w1 : w2);
+                    q[j] = (word >> (jj < 5 ? 3 * jj : 16 + 3 * (jj - 5))) & 7u;
+                } else {
+                    const int bit = i == 30 ? 15 : 31;
+                    q[j] = ((w0 >> bit) & 1u) | (((w1 >> bit) & 1u) << 1) | (((w2 >> bit) & 1u) << 2);
+                }
+            }
+        } else if (BITS == 4) {
             uint32_t w = qweight[(size_t)n * (K / 8) + k0 / 8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) q[j] = (w >> (4 * j)) & 0xFu;
@@ -174,7 +229,9 @@ dmr_status_t launch_quantize(const uint16_t *W, int N, int K, int bits, int g, u
     const int warps_per_block = 8;
     long long blocks = (items + warps_per_block - 1) / warps_per_block;
     if (blocks > 148 * 32) blocks = 148 * 32;
-    if (bits == 4)
+    if (bits == 3)
+        quantize_kernel<3><<<(int)blocks, 256, 0, st>>>(W, N, K, g, qweight, scales, zeros, dev_status);
+    else if (bits == 4)
         quantize_kernel<4><<<(int)blocks, 256, 0, st>>>(W, N, K, g, qweight, scales, zeros, dev_status);
     else
         quantize_kernel<8><<<(int)blocks, 256, 0, st>>>(W, N, K, g, qweight, scales, zeros, dev_status);
@@ -186,7 +243,12 @@ dmr_status_t launch_dequantize(const uint32_t *qweight, const uint16_t *scales, 
     const long long total = (long long)N * (K / 8);
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 64) blocks = 148 * 64;
-    if (bits == 4) {
+    if (bits == 3) {
+        if (out == DMR_OUT_F32)
+            dequantize_kernel<3, true><<<(int)blocks, 256, 0, st>>>(qweight, scales, zeros, N, K, g, W_out);
+        else
+            dequantize_kernel<3, false><<<(int)blocks, 256, 0, st>>>(qweight, scales, zeros, N, K, g, W_out);
+    } else if (bits == 4) {
         if (out == DMR_OUT_F32)
             dequantize_kernel<4, true><<<(int)blocks, 256, 0, st>>>(qweight, scales, zeros, N, K, g, W_out);
         else

@@ -11,7 +11,7 @@ namespace {
 // ---------------------------------------------------------------------------------------------
 // Any-shape fallback: one warp per output feature, fp32 FMAs, lanes stride over k in chunks of 8.
 // ---------------------------------------------------------------------------------------------
-template <int MODE /*0 dense, 4, 8*/, bool OUT_F32>
+template <int MODE /*0 dense, 3, 4, 8*/, bool OUT_F32>
 __global__ void __launch_bounds__(256)
 simple_linear_kernel(const uint16_t *__restrict__ X, int M, const int32_t *__restrict__ idx,
                      const int32_t *__restrict__ count, int coff, const void *__restrict__ Wany,
@@ -35,7 +35,23 @@ simple_linear_kernel(const uint16_t *__restrict__ X, int M, const int32_t *__res
                 const float s = __uint_as_float((uint32_t)scales[(size_t)n * G + k0 / g_size] << 16);
                 const float z = (float)zeros[(size_t)n * G + k0 / g_size];
                 const uint32_t *qp = reinterpret_cast<const uint32_t *>(Wany);
-                if (MODE == 4) {
+                if (MODE == 3) {
+                    const uint32_t *u = qp + (size_t)n * (K / 32 * 3) + (size_t)(k0 / 32) * 3;
+                    const uint32_t u0 = u[0], u1 = u[1], u2 = u[2];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int i = k0 % 32 + j;  // code i < 30: word i / 10, five codes per half-word; codes 30, 31: bits 15, 31
+                        uint32_t q;
+                        if (i < 30) {
+                            const int jj = i % 10;
+                            q = ((i < 10 ? u0 : (i < 20 ? u1 : u2)) >> (jj < 5 ? 3 * jj : 16 + 3 * (jj - 5))) & 7u;
+                        } else {
+                            const int bit = i == 30 ? 15 : 31;
+                            q = ((u0 >> bit) & 1u) | (((u1 >> bit) & 1u) << 1) | (((u2 >> bit) & 1u) << 2);
+                        }
+                        w[j] = s * ((float)q - z);
+                    }
+                } else if (MODE == 4) {
                     const uint32_t u = qp[(size_t)n * (K / 8) + k0 / 8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) w[j] = s * ((float)((u >> (4 * j)) & 0xFu) - z);
@@ -69,7 +85,12 @@ dmr_status_t launch_simple_lowbit(const uint16_t *X, int M, RowSel sel, const ui
                                   const uint16_t *scales, const uint8_t *zeros, int N, int K, int bits,
                                   int g, void *Y, dmr_out_t out, cudaStream_t st) {
     const int grid = (N + 7) / 8;
-    if (bits == 4) {
+    if (bits == 3) {
+        if (out == DMR_OUT_F32)
+            simple_linear_kernel<3, true><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+        else
+            simple_linear_kernel<3, false><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
+    } else if (bits == 4) {
         if (out == DMR_OUT_F32)
             simple_linear_kernel<4, true><<<grid, 256, 0, st>>>(X, M, sel.idx, sel.count, sel.offset, qweight, scales, zeros, N, K, g, Y);
         else

@@ -38,7 +38,8 @@ def test_size_queries(L):
     assert L.dmr_qweight_bytes(8, 256, QFormat(8, 0)) == 8 * 256
     assert L.dmr_scales_bytes(8, 256, QFormat(8, 0)) == 8 * 2
     assert L.dmr_qweight_bytes(8, 96, QFormat(4, 64)) == 0      # g does not divide K
-    assert L.dmr_qweight_bytes(8, 256, QFormat(3, 128)) == 0    # unsupported width
+    assert L.dmr_qweight_bytes(8, 256, QFormat(3, 128)) == 8 * 256 * 3 // 8   # 32 codes in three words
+    assert L.dmr_qweight_bytes(8, 256, QFormat(2, 128)) == 0    # unsupported width
     for op in (0, 1, 2):
         b = L.dmr_workspace_bytes(op, 64, 5120, 5120, f)
         assert b >= 256 and b % 256 == 0
@@ -63,7 +64,7 @@ def test_argument_errors_are_reported_before_any_launch(L):
     # null pointers / bad sizes
     assert L.dmr_quantize(None, 8, 128, f, p, p, p, None, None) == 1
     assert L.dmr_quantize(p, 8, 96, QFormat(4, 64), p, p, p, None, None) == 1
-    assert L.dmr_quantize(p, 8, 128, QFormat(3, 128), p, p, p, None, None) == 2
+    assert L.dmr_quantize(p, 8, 128, QFormat(2, 128), p, p, p, None, None) == 2
     assert L.dmr_quantize(odd, 8, 128, f, p, p, p, None, None) == 3
     assert L.dmr_lowbit_linear(p, -1, p, p, p, 8, 128, f, p, 0, p, 4096, None) == 1
     assert L.dmr_lowbit_linear(p, 1, None, p, p, 8, 128, f, p, 0, p, 4096, None) == 1
