@@ -66,6 +66,7 @@ struct DecodeArgs {
     int sz_stage;             // 1: a tile's scales and zero points are copied to shared memory ahead of time
     int sz_vec;               // 1: the entries of a box's groups are consecutive, aligned and read with one load each (shared or global)
     int sz_zoff, sz_stride;   // shared-memory offset of a tile's zero points; bytes between the tile buffers
+    int sx_off, sx_warp;      // FAST: shared-memory offset of the cached activation sums; bytes per warp
 };
 
 __device__ __forceinline__ uint4 ldg_v4(const void *p) {
@@ -87,6 +88,14 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
 __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
     uint2 v;
     asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_f32x2(uint32_t addr, float x, float y) {
+    asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(addr), "f"(x), "f"(y) : "memory");
+}
+__device__ __forceinline__ float2 lds_f32x2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
@@ -120,17 +129,21 @@ struct DecodeCfg {
     static constexpr int STAGE_BYTES = TILE * BOX_BYTES;
     static constexpr int NACC = R * NT * 4;
     static constexpr int RING_BYTES = WARPS * D * STAGE_BYTES;
-    static constexpr int RED_BUFS = WARPS * NACC * 32 * 4 * 2 <= 32 * 1024 ? 2 : 1;  // one buffer costs a second barrier per tile
+    static constexpr int RED_BUFS = 2;                         // tile t's sums are written while tile t - 1's are added up
     static constexpr int RED_BYTES = RED_BUFS * WARPS * NACC * 32 * 4;
-    static constexpr int BAR_OFF = RING_BYTES + RED_BYTES;     // WARPS * D ring barriers, then kSzBuffers table barriers
-    static constexpr int SZ_OFF = BAR_OFF + ((WARPS * D + kSzBuffers) * 8 + 15) / 16 * 16;
+    static constexpr int BAR_OFF = RING_BYTES + RED_BYTES;     // WARPS * D ring barriers, kSzBuffers table barriers, RED_BUFS sum barriers
+    static constexpr int SZ_OFF = BAR_OFF + ((WARPS * D + kSzBuffers + RED_BUFS) * 8 + 15) / 16 * 16;
     static constexpr size_t SMEM = (size_t)SZ_OFF + 1024 /*alignment slack*/;  // plus kSzBuffers * sz_stride when staging
 };
 
 // NT: 8-row activation blocks (1 or 2).  R: 16-row weight blocks per tile.  WPL: code words per lane and
 // row in one chunk (4: chunks of 128 input features, for groups that are multiples of 128; 2: chunks of
 // 64, for groups of 64).  WARPS: warps per CTA.  D: stages of a warp's ring.
-template <int BITS, int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
+// FAST: the common layer shape, fixed at compile time so that the hot loop carries no shape tests - every tile is
+// whole and its scales and zero points are staged in shared memory, a chunk is one quantization group, K is a whole
+// number of boxes, and the sums of the activations per chunk (which do not depend on the tile) fit in shared memory:
+// they are formed during the CTA's first tile and read back afterwards.
+template <int BITS, int NT, int R, int WPL, int WARPS, int D, bool OUT_F32, bool FAST>
 __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_constant__ CUtensorMap wmap, const DecodeArgs a) {
     using Cfg = DecodeCfg<BITS, NT, R, WPL, WARPS, D>;
     constexpr int TILE = Cfg::TILE, CHUNK_K = Cfg::CHUNK_K, NACC = Cfg::NACC, THREADS = Cfg::THREADS, CPB = Cfg::CPB;
@@ -147,7 +160,9 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
     const uint32_t ring = base + (uint32_t)warp * (D * Cfg::STAGE_BYTES);
     const uint32_t bars = base + Cfg::BAR_OFF + (uint32_t)warp * (D * 8);
     const uint32_t szbars = base + Cfg::BAR_OFF + WARPS * D * 8;
+    const uint32_t redbars = szbars + kSzBuffers * 8;  // "every warp has written its sums of this tile", one per buffer
     const uint32_t szbuf = base + Cfg::SZ_OFF;
+    const uint32_t sxbase = base + (uint32_t)a.sx_off + (uint32_t)(warp * a.sx_warp);  // FAST: this warp's cached activation sums
     const int nboxes = (a.nchunks + CPB - 1) / CPB;
 
     // Every warp sets up its own ring and starts its first copies at once; the barriers of the shared scale / zero-point
@@ -159,6 +174,8 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
         if (warp == 0) {
 #pragma unroll
             for (int d = 0; d < kSzBuffers; ++d) mbar_init(szbars + 8 * d, 1);
+#pragma unroll
+            for (int d = 0; d < Cfg::RED_BUFS; ++d) mbar_init(redbars + 8 * d, WARPS);
         }
         fence_barrier_init();
     }
@@ -168,7 +185,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
     // ---- a tile's scales and zero points into shared memory (two contiguous blocks of the tables) ----
     int sz_issued = 0;
     auto issue_sz = [&](int tile) {  // by thread 0; tiles in the order this CTA takes them
-        if (!a.sz_stage || tile >= t1) return;
+        if (!(FAST || a.sz_stage) || tile >= t1) return;
         const int d = sz_issued % kSzBuffers;
         const uint32_t n_entries = (uint32_t)(TILE * a.G);  // staging is only chosen when every tile is whole
         mbar_expect_tx(szbars + 8 * d, n_entries * 3);
@@ -197,8 +214,8 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
 #pragma unroll
     for (int d = 0; d < D; ++d) issue();
     if (threadIdx.x == 0) {
-        issue_sz(t0);
-        issue_sz(t0 + 1);
+#pragma unroll
+        for (int d = 0; d < kSzBuffers; ++d) issue_sz(t0 + d);
     }
     __syncthreads();  // warp 0's barriers are set up before anyone waits on them
 
@@ -243,6 +260,29 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[r][nt][c] = 0.f;
 
+    // Adds the warps' sums of tile `tile` (the CTA's tile number `tl`) in warp order and writes the outputs.
+    auto finish_tile = [&](int tile, int tl) {
+        if (ok) ok = mbar_wait(redbars + 8 * (tl & 1), (uint32_t)((tl >> 1) & 1), a.status);
+        // every warp is past that tile's table: its buffer takes the tile kSzBuffers further on
+        if (threadIdx.x == 0 && ok) issue_sz(tile + kSzBuffers);
+        const float *rbuf = red + (size_t)(tl & 1) * WARPS * (NACC * 32);
+        for (int o = threadIdx.x; o < NACC * 32; o += THREADS) {
+            const int e = o >> 5, l = o & 31;
+            float v = rbuf[e * 32 + l];
+#pragma unroll
+            for (int w2 = 1; w2 < WARPS; ++w2) v += rbuf[(w2 * NACC + e) * 32 + l];
+            const int c = e & 3, nt = (e >> 2) % NT, r = (e >> 2) / NT;
+            const int slot = nt * 8 + 2 * (l & 3) + (c & 1);
+            const int lg = l >> 2;
+            const int n = tile * TILE + r * 16 + (BITS == 3 ? lg : ((lg >> 1) | ((lg & 1) << 2))) + 8 * (c >> 1);
+            if (ok && slot < rows && n < a.N) {
+                const int row = a.idx ? a.idx[slot] : slot;
+                if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
+                else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
+            }
+        }
+    };
+
     int consumed = 0;
     constexpr uint32_t kOnes = 0x3F803F80u;  // bf16 1.0 twice
     for (int tile = t0, tl = 0; tile < t1; ++tile, ++tl) {
@@ -253,26 +293,27 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int n = min(tile * TILE + pg + r * 16 + h * 8, a.N - 1);
-                szo[r][h] = (uint32_t)(a.sz_stage ? n - tile * TILE : n) * (uint32_t)a.G;
+                szo[r][h] = (uint32_t)((FAST || a.sz_stage) ? n - tile * TILE : n) * (uint32_t)a.G;
             }
         const uint32_t sbase = szbuf + (uint32_t)(tl % kSzBuffers) * a.sz_stride, zbase = sbase + a.sz_zoff;
-        if (a.sz_stage && ok) ok = mbar_wait(szbars + 8 * (tl % kSzBuffers), (uint32_t)((tl / kSzBuffers) & 1), a.status);
-        for (int box = warp; box < nboxes; box += WARPS) {
+        if ((FAST || a.sz_stage) && ok) ok = mbar_wait(szbars + 8 * (tl % kSzBuffers), (uint32_t)((tl / kSzBuffers) & 1), a.status);
+        const bool form_sx = !FAST || tl == 0;  // FAST: the activation sums are formed in the first tile and kept
+        for (int box = warp, bl = 0; box < nboxes; box += WARPS, ++bl) {
             const int d = consumed % D;
             if (ok) ok = mbar_wait(bars + 8 * d, (uint32_t)((consumed / D) & 1), a.status);
             ++consumed;
             const uint32_t stage = ring + d * Cfg::STAGE_BYTES;
-            const int nsub = min(CPB, a.nchunks - box * CPB);
+            const int nsub = FAST ? CPB : min(CPB, a.nchunks - box * CPB);
             const int grp0 = a.g_shift >= 0 ? ((box * CPB * CHUNK_K) >> a.g_shift) : ((box * CPB * CHUNK_K) / a.g_size);
             // scales and zero points of the box's groups when they sit side by side in the tile's copy
             uint32_t scv[R][2][CPB / 2], zpv[R][2];
-            if (a.sz_vec) {
+            if (FAST || a.sz_vec) {
 #pragma unroll
                 for (int r = 0; r < R; ++r)
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const uint32_t o = szo[r][h] + (uint32_t)grp0;
-                        if (a.sz_stage) {
+                        if (FAST || a.sz_stage) {
                             if constexpr (CPB == 2) {
                                 scv[r][h][0] = lds_u32(sbase + 2 * o);
                                 zpv[r][h] = lds_u16(zbase + o);
@@ -297,11 +338,11 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
             }
 #pragma unroll(NT == 1 ? CPB : 1)
             for (int sub = 0; sub < CPB; ++sub) {
-                if (sub >= nsub) break;
+                if (!FAST && sub >= nsub) break;
                 const int chunk = box * CPB + sub;
                 // scale (as fp32 bits) and zero point of this chunk's group for the lane's rows
                 uint32_t sc[R][2], zp[R][2];
-                if (a.sz_vec) {
+                if (FAST || a.sz_vec) {
 #pragma unroll
                     for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -327,6 +368,15 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                         }
                 }
                 float gs[R][NT][4], sx[NT][4];
+                const uint32_t sxaddr = sxbase + (uint32_t)(((bl * CPB + sub) * NT) * 256 + lane * 8);
+                if (FAST && !form_sx) {
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const float2 v = lds_f32x2(sxaddr + nt * 256);
+                        sx[nt][0] = sx[nt][2] = v.x;
+                        sx[nt][1] = sx[nt][3] = v.y;
+                    }
+                }
                 if constexpr (BITS == 3) {
                     // Lane (g, t) takes block t of the chunk (32 codes in three words) for rows g and g + 8 of each 16-row
                     // block, and the 32 activations they meet.
@@ -360,8 +410,10 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                                                     ((hi & 1) ? 0x7600u : 0x5400u) | ((lo & 1) ? 0x32u : 0x10u));
                                 }
                             }
-                            if (mi == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
-                            else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                            if (form_sx) {
+                                if (mi == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                                else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                            }
                         }
 #pragma unroll
                         for (int r = 0; r < R; ++r) {
@@ -428,9 +480,11 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                         b[nt][1] = prmt(x[nt][j][0], x[nt][j][2], 0x7632);
                         b[nt][2] = prmt(x[nt][j][1], x[nt][j][3], 0x5410);
                         b[nt][3] = prmt(x[nt][j][1], x[nt][j][3], 0x7632);
-                        if (j == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
-                        else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
-                        mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][2], b[nt][3]);
+                        if (form_sx) {
+                            if (j == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                            else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
+                            mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][2], b[nt][3]);
+                        }
                     }
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
@@ -473,6 +527,10 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                     }
                     if (more) load_x(nc);
                 }
+                if (FAST && form_sx) {
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) sts_f32x2(sxaddr + nt * 256, sx[nt][0], sx[nt][1]);
+                }
                 // the chunk lies inside one quantization group: s (sum x (128 + q) - (128 + z) sum x)
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
@@ -488,8 +546,12 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                 }
             }
         }
-        // ---- end of a tile: add the warps' sums in warp order and write the outputs ----
-        float *rbuf = red + (size_t)(Cfg::RED_BUFS == 2 ? (tl & 1) : 0) * WARPS * (NACC * 32);
+        // ---- end of a tile.  No CTA-wide barrier: a warp first adds up and writes the outputs of the tile BEFORE (all
+        // warps have announced their sums of that one, normally long ago), then puts its own sums of this tile into
+        // the other buffer and announces them.  A warp can so run up to one tile ahead of the slowest one, and the
+        // buffer it writes is free: whoever announced tile t had finished reading tile t - 1 before.
+        if (tl > 0) finish_tile(tile - 1, tl - 1);
+        float *rbuf = red + (size_t)(tl & 1) * WARPS * (NACC * 32);
 #pragma unroll
         for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -499,26 +561,10 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                     rbuf[(warp * NACC + (r * NT + nt) * 4 + c) * 32 + lane] = acc[r][nt][c];
                     acc[r][nt][c] = 0.f;
                 }
-        __syncthreads();
-        // every warp is past this tile's table: its buffer takes the tile kSzBuffers - 1 further on
-        if (threadIdx.x == 0 && ok) issue_sz(tile + kSzBuffers - 1);
-        for (int o = threadIdx.x; o < NACC * 32; o += THREADS) {
-            const int e = o >> 5, l = o & 31;
-            float v = rbuf[e * 32 + l];
-#pragma unroll
-            for (int w2 = 1; w2 < WARPS; ++w2) v += rbuf[(w2 * NACC + e) * 32 + l];
-            const int c = e & 3, nt = (e >> 2) % NT, r = (e >> 2) / NT;
-            const int slot = nt * 8 + 2 * (l & 3) + (c & 1);
-            const int lg = l >> 2;
-            const int n = tile * TILE + r * 16 + (BITS == 3 ? lg : ((lg >> 1) | ((lg & 1) << 2))) + 8 * (c >> 1);
-            if (ok && slot < rows && n < a.N) {
-                const int row = a.idx ? a.idx[slot] : slot;
-                if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
-                else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
-            }
-        }
-        if (Cfg::RED_BUFS == 1) __syncthreads();  // the sums are read before the next tile's overwrite them
+        __syncwarp();
+        if (lane == 0) mbar_arrive(redbars + 8 * (tl & 1));
     }
+    finish_tile(t1 - 1, t1 - 1 - t0);
 }
 
 int device_sm_count() {
@@ -542,39 +588,13 @@ bool decode_pdl_enabled() {
     return v != 0;
 }
 
-template <int BITS, int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
-dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
-    using Cfg = DecodeCfg<BITS, NT, R, WPL, WARPS, D>;
-    constexpr int TILE = Cfg::TILE;
-    // shared memory left for the copies of the scale / zero-point tables (227 KB per CTA at most)
-    constexpr size_t kSzBudget = 227 * 1024 - Cfg::SMEM < 36 * 1024 ? 227 * 1024 - Cfg::SMEM : 36 * 1024;
-    static_assert(Cfg::SMEM <= 227 * 1024, "ring and reduction buffers exceed an SM's shared memory");
-    auto kernel = decode_w4_kernel<BITS, NT, R, WPL, WARPS, D, OUT_F32>;
-    if (!ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), Cfg::SMEM + kSzBudget < kMinSmem ? kMinSmem : Cfg::SMEM + kSzBudget))
-        return DMR_ERR_CUDA;
-    a.tiles = (a.N + TILE - 1) / TILE;
-    a.nchunks = a.K / Cfg::CHUNK_K;
-    int ctas = device_sm_count();
-    if (ctas > a.tiles) ctas = a.tiles;
-    // A tile's scales and zero points are two contiguous blocks of the tables: they are copied to shared memory ahead
-    // of time when every tile is whole, the blocks are 16-byte aligned and three tiles' worth stay small.
-    const size_t tile_entries = (size_t)TILE * a.G;
-    a.sz_zoff = (int)((tile_entries * 2 + 15) / 16 * 16);
-    a.sz_stride = a.sz_zoff + (int)((tile_entries + 15) / 16 * 16);
-    a.sz_stage = (a.N % TILE == 0 && tile_entries % 16 == 0 && ((uintptr_t)a.scales % 16) == 0 && ((uintptr_t)a.zeros % 16) == 0 &&
-                  (size_t)kSzBuffers * a.sz_stride <= kSzBudget) ? 1 : 0;
-    // a box covers CPB consecutive groups and every row's entries start at a multiple of CPB
-    a.sz_vec = (a.g_size == Cfg::CHUNK_K && a.G % Cfg::CPB == 0 &&
-                (a.sz_stage || (((uintptr_t)a.scales % (2 * Cfg::CPB)) == 0 && ((uintptr_t)a.zeros % Cfg::CPB) == 0))) ? 1 : 0;
-    const size_t smem = Cfg::SMEM + (a.sz_stage ? (size_t)kSzBuffers * a.sz_stride : 0);
-    CUtensorMap wmap;
-    const uint64_t rb = (uint64_t)a.K * BITS / 8;
-    if (!make_tensor_map_2d(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.qweight, (uint64_t)a.N, rb, rb, TILE, Cfg::BOX_BYTES,
-                            BITS == 3 ? TmaSwizzle::kNone : TmaSwizzle::k128B))
-        return DMR_ERR_CUDA;
+template <int BITS, int NT, int R, int WPL, int WARPS, int D, bool OUT_F32, bool FAST>
+dmr_status_t launch_decode_k(const DecodeArgs &a, const CUtensorMap &wmap, int ctas, size_t smem, size_t smem_attr, cudaStream_t st) {
+    auto kernel = decode_w4_kernel<BITS, NT, R, WPL, WARPS, D, OUT_F32, FAST>;
+    if (!ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), smem_attr)) return DMR_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas, 1, 1);
-    cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
+    cfg.blockDim = dim3(WARPS * 32, 1, 1);
     // more than half of an SM's shared memory: two CTAs of these kernels never share an SM (see above)
     cfg.dynamicSmemBytes = smem < kMinSmem ? kMinSmem : smem;
     cfg.stream = st;
@@ -594,6 +614,46 @@ dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
         return DMR_ERR_CUDA;
     }
     return check_launch();
+}
+
+template <int BITS, int NT, int R, int WPL, int WARPS, int D, bool OUT_F32>
+dmr_status_t launch_decode_t(DecodeArgs a, cudaStream_t st) {
+    using Cfg = DecodeCfg<BITS, NT, R, WPL, WARPS, D>;
+    constexpr int TILE = Cfg::TILE;
+    // shared memory left for the copies of the scale / zero-point tables (227 KB per CTA at most)
+    constexpr size_t kSzBudget = 227 * 1024 - Cfg::SMEM < 36 * 1024 ? 227 * 1024 - Cfg::SMEM : 36 * 1024;
+    static_assert(Cfg::SMEM <= 227 * 1024, "ring and reduction buffers exceed an SM's shared memory");
+    constexpr size_t kSmemMax = 227 * 1024;
+    constexpr size_t smem_attr = Cfg::SMEM + kSzBudget < kMinSmem ? kMinSmem : Cfg::SMEM + kSzBudget;
+    a.tiles = (a.N + TILE - 1) / TILE;
+    a.nchunks = a.K / Cfg::CHUNK_K;
+    int ctas = device_sm_count();
+    if (ctas > a.tiles) ctas = a.tiles;
+    // A tile's scales and zero points are two contiguous blocks of the tables: they are copied to shared memory ahead
+    // of time when every tile is whole, the blocks are 16-byte aligned and three tiles' worth stay small.
+    const size_t tile_entries = (size_t)TILE * a.G;
+    a.sz_zoff = (int)((tile_entries * 2 + 15) / 16 * 16);
+    a.sz_stride = a.sz_zoff + (int)((tile_entries + 15) / 16 * 16);
+    a.sz_stage = (a.N % TILE == 0 && tile_entries % 16 == 0 && ((uintptr_t)a.scales % 16) == 0 && ((uintptr_t)a.zeros % 16) == 0 &&
+                  (size_t)kSzBuffers * a.sz_stride <= kSzBudget) ? 1 : 0;
+    // a box covers CPB consecutive groups and every row's entries start at a multiple of CPB
+    a.sz_vec = (a.g_size == Cfg::CHUNK_K && a.G % Cfg::CPB == 0 &&
+                (a.sz_stage || (((uintptr_t)a.scales % (2 * Cfg::CPB)) == 0 && ((uintptr_t)a.zeros % Cfg::CPB) == 0))) ? 1 : 0;
+    size_t smem = Cfg::SMEM + (a.sz_stage ? (size_t)kSzBuffers * a.sz_stride : 0);
+    // FAST: the sums of the activations per chunk and batch column, kept from the CTA's first tile on (8 bytes per lane)
+    const int nboxes = (a.nchunks + Cfg::CPB - 1) / Cfg::CPB;
+    a.sx_off = (int)((smem - 1024 + 15) / 16 * 16);
+    a.sx_warp = (nboxes + WARPS - 1) / WARPS * Cfg::CPB * NT * 256;
+    const size_t smem_fast = (size_t)a.sx_off + (size_t)WARPS * a.sx_warp + 1024;
+    const bool fast = a.sz_stage && a.sz_vec && a.nchunks % Cfg::CPB == 0 && smem_fast <= kSmemMax;
+    if (fast) smem = smem_fast;
+    CUtensorMap wmap;
+    const uint64_t rb = (uint64_t)a.K * BITS / 8;
+    if (!make_tensor_map_2d(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.qweight, (uint64_t)a.N, rb, rb, TILE, Cfg::BOX_BYTES,
+                            BITS == 3 ? TmaSwizzle::kNone : TmaSwizzle::k128B))
+        return DMR_ERR_CUDA;
+    return fast ? launch_decode_k<BITS, NT, R, WPL, WARPS, D, OUT_F32, true>(a, wmap, ctas, smem, kSmemMax, st)
+                : launch_decode_k<BITS, NT, R, WPL, WARPS, D, OUT_F32, false>(a, wmap, ctas, smem, smem_attr, st);
 }
 
 }  // namespace
