@@ -155,6 +155,8 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
     const int g = lane >> 2, t = lane & 3;
     // box row of fragment row g: 0, 4, 1, 5, ... for 4-bit codes (bank-conflict-free under the swizzle); 3-bit boxes are not swizzled
     const int pg = BITS == 3 ? g : ((g >> 1) | ((g & 1) << 2));
+    // 4-bit codes: where this lane's words of fragment row g and chunk 0 sit inside a stage
+    const uint32_t lane_off = (uint32_t)(pg * Cfg::BOX_BYTES) + (WPL == 4 ? (uint32_t)((t ^ pg) << 4) : (uint32_t)((((t >> 1) ^ pg) << 4) + (t & 1) * 8));
     const int t0 = (int)(((long long)blockIdx.x * a.tiles) / gridDim.x);
     const int t1 = (int)(((long long)(blockIdx.x + 1) * a.tiles) / gridDim.x);
     const uint32_t ring = base + (uint32_t)warp * (D * Cfg::STAGE_BYTES);
@@ -251,6 +253,16 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
             }
     };
     if (has_boxes) load_x(warp * CPB);
+    // B fragments: the chunk's activations paired like the codes.  4-bit word j: (x0, x4), (x1, x5), (x2, x6), (x3, x7);
+    // 3-bit block: pair p = 5 j + i is (x[10 j + i], x[10 j + i + 5]), pair 15 is (x30, x31).
+    auto xfrag4 = [&](int nt, int j, int q) -> uint32_t {
+        return prmt(x[nt][j][q >> 1], x[nt][j][(q >> 1) + 2], (q & 1) ? 0x7632u : 0x5410u);
+    };
+    auto xfrag3 = [&](int nt, int p) -> uint32_t {
+        if (p == 15) return x[nt][3][3];
+        const int lo = 10 * (p / 5) + p % 5, hi = lo + 5;  // activations 2 v, 2 v + 1 are in word v
+        return prmt(x[nt][lo >> 3][(lo >> 1) & 3], x[nt][hi >> 3][(hi >> 1) & 3], ((hi & 1) ? 0x7600u : 0x5400u) | ((lo & 1) ? 0x32u : 0x10u));
+    };
 
     float acc[R][NT][4];
 #pragma unroll
@@ -268,14 +280,15 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
         const float *rbuf = red + (size_t)(tl & 1) * WARPS * (NACC * 32);
         for (int o = threadIdx.x; o < NACC * 32; o += THREADS) {
             const int e = o >> 5, l = o & 31;
+            const int c = e & 3, nt = (e >> 2) % NT, r = (e >> 2) / NT;
+            const int slot = nt * 8 + 2 * (l & 3) + (c & 1);
+            if (slot >= rows) continue;  // a batch column nobody asked for
             float v = rbuf[e * 32 + l];
 #pragma unroll
             for (int w2 = 1; w2 < WARPS; ++w2) v += rbuf[(w2 * NACC + e) * 32 + l];
-            const int c = e & 3, nt = (e >> 2) % NT, r = (e >> 2) / NT;
-            const int slot = nt * 8 + 2 * (l & 3) + (c & 1);
             const int lg = l >> 2;
             const int n = tile * TILE + r * 16 + (BITS == 3 ? lg : ((lg >> 1) | ((lg & 1) << 2))) + 8 * (c >> 1);
-            if (ok && slot < rows && n < a.N) {
+            if (ok && n < a.N) {
                 const int row = a.idx ? a.idx[slot] : slot;
                 if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
                 else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
@@ -304,7 +317,8 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
             ++consumed;
             const uint32_t stage = ring + d * Cfg::STAGE_BYTES;
             const int nsub = FAST ? CPB : min(CPB, a.nchunks - box * CPB);
-            const int grp0 = a.g_shift >= 0 ? ((box * CPB * CHUNK_K) >> a.g_shift) : ((box * CPB * CHUNK_K) / a.g_size);
+            const int grp0 = FAST ? box * CPB  // a chunk is a group
+                                  : (a.g_shift >= 0 ? ((box * CPB * CHUNK_K) >> a.g_shift) : ((box * CPB * CHUNK_K) / a.g_size));
             // scales and zero points of the box's groups when they sit side by side in the tile's copy
             uint32_t scv[R][2][CPB / 2], zpv[R][2];
             if (FAST || a.sz_vec) {
@@ -336,11 +350,11 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                         }
                     }
             }
-#pragma unroll(NT == 1 ? CPB : 1)
+#pragma unroll
             for (int sub = 0; sub < CPB; ++sub) {
                 if (!FAST && sub >= nsub) break;
                 const int chunk = box * CPB + sub;
-                // scale (as fp32 bits) and zero point of this chunk's group for the lane's rows
+                // scale and 128 + zero point (both as fp32 bits) of this chunk's group for the lane's rows
                 uint32_t sc[R][2], zp[R][2];
                 if (FAST || a.sz_vec) {
 #pragma unroll
@@ -349,7 +363,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                         for (int h = 0; h < 2; ++h) {
                             const uint32_t pair = scv[r][h][sub / 2];
                             sc[r][h] = (sub & 1) ? (pair & 0xFFFF0000u) : (pair << 16);
-                            zp[r][h] = (zpv[r][h] >> (8 * sub)) & 0xFFu;
+                            zp[r][h] = prmt(zpv[r][h], 0x00004300u, 0x5044u | ((uint32_t)sub << 8));  // fp32 bits of 128 + z
                         }
                 } else {
                     const int k0 = chunk * CHUNK_K;
@@ -360,21 +374,35 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                         for (int h = 0; h < 2; ++h) {
                             if (a.sz_stage) {
                                 sc[r][h] = lds_u16(sbase + 2 * (szo[r][h] + grp)) << 16;
-                                zp[r][h] = lds_u8(zbase + szo[r][h] + grp);
+                                zp[r][h] = (lds_u8(zbase + szo[r][h] + grp) | 0x4300u) << 16;
                             } else {
                                 sc[r][h] = (uint32_t)__ldg(a.scales + szo[r][h] + grp) << 16;
-                                zp[r][h] = __ldg(a.zeros + szo[r][h] + grp);
+                                zp[r][h] = ((uint32_t)__ldg(a.zeros + szo[r][h] + grp) | 0x4300u) << 16;
                             }
                         }
                 }
                 float gs[R][NT][4], sx[NT][4];
                 const uint32_t sxaddr = sxbase + (uint32_t)(((bl * CPB + sub) * NT) * 256 + lane * 8);
-                if (FAST && !form_sx) {
+                if constexpr (FAST) {
+                    if (form_sx) {  // the CTA's first tile: an all-ones operand against every B fragment of the chunk
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        const float2 v = lds_f32x2(sxaddr + nt * 256);
-                        sx[nt][0] = sx[nt][2] = v.x;
-                        sx[nt][1] = sx[nt][3] = v.y;
+                        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+                            for (int m = 0; m < 2 * WPL; ++m) {
+                                const uint32_t b0 = BITS == 3 ? xfrag3(nt, 2 * m) : xfrag4(nt, m >> 1, 2 * (m & 1));
+                                const uint32_t b1 = BITS == 3 ? xfrag3(nt, 2 * m + 1) : xfrag4(nt, m >> 1, 2 * (m & 1) + 1);
+                                if (m == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b0, b1);
+                                else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b0, b1);
+                            }
+                            sts_f32x2(sxaddr + nt * 256, sx[nt][0], sx[nt][1]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const float2 v = lds_f32x2(sxaddr + nt * 256);
+                            sx[nt][0] = sx[nt][2] = v.x;
+                            sx[nt][1] = sx[nt][3] = v.y;
+                        }
                     }
                 }
                 if constexpr (BITS == 3) {
@@ -399,18 +427,9 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                         uint32_t b[NT][2];
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-                            for (int q = 0; q < 2; ++q) {
-                                const int p = 2 * m + q;
-                                if (p == 15) {
-                                    b[nt][q] = x[nt][3][3];
-                                } else {
-                                    const int lo = 10 * (p / 5) + p % 5, hi = lo + 5;  // activations 2 v, 2 v + 1 are in word v
-                                    b[nt][q] = prmt(x[nt][lo >> 3][(lo >> 1) & 3], x[nt][hi >> 3][(hi >> 1) & 3],
-                                                    ((hi & 1) ? 0x7600u : 0x5400u) | ((lo & 1) ? 0x32u : 0x10u));
-                                }
-                            }
-                            if (form_sx) {
+                            b[nt][0] = xfrag3(nt, 2 * m);
+                            b[nt][1] = xfrag3(nt, 2 * m + 1);
+                            if constexpr (!FAST) {
                                 if (mi == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
                                 else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
                             }
@@ -457,15 +476,17 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                 for (int r = 0; r < R; ++r)
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const uint32_t rowaddr = stage + (uint32_t)((r * 16 + h * 8 + pg) * Cfg::BOX_BYTES);
+                        // this lane's 16 bytes of row pg under the 128-byte swizzle: chunk `sub` flips bits of the
+                        // 16-byte column index, the other rows of the fragment are whole kilobytes away
+                        const uint32_t rowaddr = ((stage + lane_off) ^ (uint32_t)(sub << (WPL == 4 ? 6 : 5))) + (uint32_t)((r * 16 + h * 8) * Cfg::BOX_BYTES);
                         if constexpr (WPL == 4) {
-                            const uint4 v = lds_v4(rowaddr + (uint32_t)(((sub * 4 + t) ^ pg) << 4));
+                            const uint4 v = lds_v4(rowaddr);
                             w[r][h][0] = v.x;
                             w[r][h][1] = v.y;
                             w[r][h][2 % WPL] = v.z;
                             w[r][h][3 % WPL] = v.w;
                         } else {
-                            const uint2 v = lds_v2(rowaddr + (uint32_t)((((sub * 2 + (t >> 1)) ^ pg) << 4) + (t & 1) * 8));
+                            const uint2 v = lds_v2(rowaddr);
                             w[r][h][0] = v.x;
                             w[r][h][1] = v.y;
                         }
@@ -476,11 +497,9 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                     uint32_t b[NT][4];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
-                        b[nt][0] = prmt(x[nt][j][0], x[nt][j][2], 0x5410);
-                        b[nt][1] = prmt(x[nt][j][0], x[nt][j][2], 0x7632);
-                        b[nt][2] = prmt(x[nt][j][1], x[nt][j][3], 0x5410);
-                        b[nt][3] = prmt(x[nt][j][1], x[nt][j][3], 0x7632);
-                        if (form_sx) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) b[nt][q] = xfrag4(nt, j, q);
+                        if constexpr (!FAST) {
                             if (j == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
                             else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
                             mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][2], b[nt][3]);
@@ -515,27 +534,13 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                 }
                 }  // 4-bit codes
                 // the next chunk's activations
-                {
-                    int nc = chunk + 1;
-                    bool more = true;
-                    if (sub == nsub - 1) {
-                        if (box + WARPS < nboxes) nc = (box + WARPS) * CPB;
-                        else {
-                            nc = warp * CPB;
-                            more = tile + 1 < t1;
-                        }
-                    }
-                    if (more) load_x(nc);
-                }
-                if (FAST && form_sx) {
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) sts_f32x2(sxaddr + nt * 256, sx[nt][0], sx[nt][1]);
-                }
+                // (after the CTA's last chunk this reads the warp's first chunk once more: always a valid address)
+                load_x(sub == nsub - 1 ? (box + WARPS < nboxes ? box + WARPS : warp) * CPB : chunk + 1);
                 // the chunk lies inside one quantization group: s (sum x (128 + q) - (128 + z) sum x)
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     const float s0 = __uint_as_float(sc[r][0]), s1 = __uint_as_float(sc[r][1]);
-                    const float z0 = __uint_as_float((zp[r][0] | 0x4300u) << 16), z1 = __uint_as_float((zp[r][1] | 0x4300u) << 16);
+                    const float z0 = __uint_as_float(zp[r][0]), z1 = __uint_as_float(zp[r][1]);
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
                         acc[r][nt][0] = fmaf(s0, fmaf(-z0, sx[nt][0], gs[r][nt][0]), acc[r][nt][0]);

@@ -9,12 +9,12 @@
 // Per 64-wide k block and stage of the ring:
 //   warp 0      TMA: the packed code tile [128 features x 32 or 64 bytes] and the activation tile
 //               [BN rows x 128 bytes, 128-byte swizzle] land in shared memory (one mbarrier);
-//   warps 2..5  one thread per feature row turns its codes into the fp16 weights s' * (q - zero)
+//   warps 2..9  two threads per feature row turn its codes into the fp16 weights s' * (q - zero)
 //               (exact integer q - zero, then ONE rounding of the product to 11 significant bits)
 //               and stores them as the swizzled K-major A tile;
 //   warp 1      one lane issues four tcgen05.mma (128 x BN x 16) that accumulate into one of two
 //               fp32 accumulators in tensor memory, and commits the stage back to the producer;
-//   warps 6..9  drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
+//   warps 10..13 drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
 //               next tile's MMAs run into the other accumulator.
 // CTAs are persistent: CTA b takes tiles b, b + grid, ...  Every wait is bounded.
 //
@@ -35,6 +35,7 @@ namespace {
 
 constexpr int PM = 128;  // features per tile (MMA M)
 constexpr int PK = 64;   // k per stage
+constexpr int UW = 8;    // unpack warps: UW / 4 groups of four, group i takes every (UW / 4)-th stage of the ring
 
 template <int BITS, int BN>
 struct PrefillCfg {
@@ -46,7 +47,7 @@ struct PrefillCfg {
     static constexpr int S_RAW = (212 * 1024) / STAGE;
     static constexpr int S = S_RAW > 8 ? 8 : S_RAW;
     static constexpr int TMEM_COLS = 2 * BN;                 // two accumulators
-    static constexpr int THREADS = 320;
+    static constexpr int THREADS = 32 * (2 + UW + 4);
     static constexpr size_t SMEM = (size_t)S * STAGE + 1024 /*alignment*/ + 512 /*barriers*/;
 };
 
@@ -164,7 +165,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         for (int s = 0; s < S; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), 1);
-            mbar_init(ready_bar(s), 4);   // one arrival per unpack warp
+            mbar_init(ready_bar(s), 4);   // one arrival per warp of the group that unpacks the stage
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull_bar(b), 1);
@@ -238,13 +239,19 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (ok) umma_commit(tfull_bar(buf));
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + UW) {
         // ================= unpack warps: codes -> fp16 weights s' * (q - zero) =================
-        const int r = (warp - 2) * 32 + lane;  // feature row of the tile
+        // A stage's chain (wait, load, convert, store, fence, arrive) is a string of shared-memory round trips that
+        // one group of four warps cannot overlap with itself, so NG groups work on different stages of the ring
+        // at the same time: group i takes the stages whose running number is i modulo NG.
+        const int r = ((warp - 2) & 3) * 32 + lane;  // feature row of the tile
+        constexpr int NG = UW / 4;
+        constexpr int CH = 8, c_lo = 0;               // 16-byte chunks (8 weights each) per thread and stage
+        const int grp_id = (warp - 2) >> 2;
         const uint32_t swz = (uint32_t)(r & 7);
-        uint32_t it = 0;
+        uint32_t it0 = 0;  // running number of the tile's first stage
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, it0 += (uint32_t)nkb) {
             const int n = min((tile % a.n_tiles) * PM + r, a.N - 1);
             const uint16_t *sp = a.scales + (size_t)n * G;
             const uint8_t *zp = a.zeros + (size_t)n * G;
@@ -254,13 +261,19 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             int fb = (int)(smax >> 7);
             fb = fb < 1 ? 1 : (fb > 253 ? 253 : fb);
             const float fdown = __uint_as_float((uint32_t)(254 - fb) << 23);  // 2^-(fb - 127)
-            uint32_t sb = __ldg(sp), zb = __ldg(zp);
-            for (int kb = 0; kb < nkb; ++kb, ++it) {
+            int kb = (int)(((uint32_t)grp_id + (uint32_t)NG - it0 % (uint32_t)NG) % (uint32_t)NG);  // this group's first k block of the tile
+            uint32_t sb = 0, zb = 0;
+            if (kb < nkb) {
+                sb = __ldg(sp + kb / kb_per_group);
+                zb = __ldg(zp + kb / kb_per_group);
+            }
+            for (; kb < nkb; kb += NG) {
+                const uint32_t it = it0 + (uint32_t)kb;
                 const int s = it % S;
-                // scale / zero of the next k block's group, fetched while this block is unpacked
+                // scale / zero of this group's next k block, fetched while this block is unpacked
                 uint32_t sb_next = sb, zb_next = zb;
-                if (kb + 1 < nkb && (kb + 1) % kb_per_group == 0) {
-                    const int grp = (kb + 1) / kb_per_group;
+                if (kb + NG < nkb) {
+                    const int grp = (kb + NG) / kb_per_group;
                     sb_next = __ldg(sp + grp);
                     zb_next = __ldg(zp + grp);
                 }
@@ -271,9 +284,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const uint32_t src = p_tile(s) + r * Cfg::P_ROW;
                 const uint32_t dst = a_tile(s) + r * 128;
                 if (BITS == 4) {
-                    uint32_t w[8];
-                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(src));
-                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "r"(src + 16));
+                    uint32_t w[CH];
+#pragma unroll
+                    for (int c4 = 0; c4 < CH; c4 += 4)
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                     : "=r"(w[c4]), "=r"(w[c4 + 1]), "=r"(w[c4 + 2]), "=r"(w[c4 + 3])
+                                     : "r"(src + 4 * (c_lo + c4)));
                     // fp16 patterns: 0x6400 | q = 1024 + q and 0x6400 | (q << 4) = 1024 + 16 q (no shift needed
                     // for the odd codes); minus 1024 + zero (or 1024 + 16 zero) is exact; then one rounding
                     const float sf = __uint_as_float(sb << 16) * fdown;
@@ -283,10 +299,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     const uint32_t zz = 0x6400u | zb, zz16 = 0x6400u | (zb << 4);
                     const uint32_t zoff = zz | (zz << 16), zoff16 = zz16 | (zz16 << 16);
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {  // word c = codes 8c .. 8c+7 = 16-byte chunk c of the row
-                        const uint32_t w8 = w[c] >> 8;
-                        const uint32_t d04 = f16x2_mul(f16x2_sub(lop3_and_or(w[c], 0x000F000Fu, 0x64006400u), zoff), s2);
-                        const uint32_t d15 = f16x2_mul(f16x2_sub(lop3_and_or(w[c], 0x00F000F0u, 0x64006400u), zoff16), s2_16);
+                    for (int cc = 0; cc < CH; ++cc) {  // word c = codes 8c .. 8c+7 = 16-byte chunk c of the row
+                        const int c = c_lo + cc;
+                        const uint32_t w8 = w[cc] >> 8;
+                        const uint32_t d04 = f16x2_mul(f16x2_sub(lop3_and_or(w[cc], 0x000F000Fu, 0x64006400u), zoff), s2);
+                        const uint32_t d15 = f16x2_mul(f16x2_sub(lop3_and_or(w[cc], 0x00F000F0u, 0x64006400u), zoff16), s2_16);
                         const uint32_t d26 = f16x2_mul(f16x2_sub(lop3_and_or(w8, 0x000F000Fu, 0x64006400u), zoff), s2);
                         const uint32_t d37 = f16x2_mul(f16x2_sub(lop3_and_or(w8, 0x00F000F0u, 0x64006400u), zoff16), s2_16);
                         const uint32_t o01 = prmt(d04, d15, 0x5410), o45 = prmt(d04, d15, 0x7632);
@@ -298,7 +315,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     const float zf = __uint_as_float(0x4B000000u | zb);  // 2^23 + zero
                     const float sf = __uint_as_float(sb << 16) * fdown;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {  // chunk c = codes 8c .. 8c+7 = packed words 2c, 2c+1
+                    for (int cc = 0; cc < CH; ++cc) {  // chunk c = codes 8c .. 8c+7 = packed words 2c, 2c+1
+                        const int c = c_lo + cc;
                         uint32_t w0, w1;
                         asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w0), "=r"(w1) : "r"(src + 8 * c));
                         uint32_t o[4];
