@@ -36,7 +36,7 @@ DECODE_MS = (1, 8, 16)
 BITS, GROUP = 4, 128
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of decode_w4_kernel, mean of the four 7B-class
 # linears at M = 1 (ncu capture summarised in profiles/decode_w4_kernel_int4_g128_7b_M1.txt)
-DECODE_TRAFFIC_BYTES_PER_LAUNCH = 26.55e6
+DECODE_TRAFFIC_BYTES_PER_LAUNCH = 26.54e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

@@ -8,7 +8,8 @@
  *     serves that step.
  *   - Sec. 5 "Experimental Models and Precision" and App. "Quantization Detail": the
  *     low-precision model is W4A16 weight-only quantization of every decoder Linear layer
- *     (activations stay 16 bit); the high-precision reference is bf16.
+ *     (activations stay 16 bit), with a W3A16 group-128 variant as the most aggressive cell; the
+ *     high-precision reference is bf16.
  *   - Sec. 4.2 "KL-to-Classification Mapping": label 1 means the step needs high precision.
  * The paper fixes no quantization arithmetic; the scheme implemented here is round-to-nearest
  * asymmetric min/max quantization with an integer zero point and a bf16 scale per group of
@@ -20,6 +21,13 @@
  *   Y  [M][N] bf16 or fp32, row-major
  *   qweight [N][K*bits/32] uint32.  bits = 4: code k of a row is in word k/8, bits 4*(k%8)..+3.
  *                                   bits = 8: code k is in word k/4, bits 8*(k%4)..+7.
+ *                                   bits = 3: every 32 codes take three words.  Code i < 30 of the block is
+ *                                   in word i/10, at bits 3*(i%10)..+2 for i%10 < 5 and at bits
+ *                                   16+3*(i%10-5)..+2 otherwise (five codes per half-word; bits 15 and 31
+ *                                   stay free); bit b of code 30 is bit 15 of word b, bit b of code 31 is
+ *                                   bit 31 of word b.  (The paper serves its 3-bit checkpoint expanded to
+ *                                   fp16 and gives no packed layout; this one is the library's own: a
+ *                                   half-word holds five codes that one mask turns into bf16 values.)
  *                                   Codes are unsigned, 0 .. 2^bits-1.
  *   scales  [N][G] bf16, zeros [N][G] uint8, G = K / g, g = group_size (0 means g = K).
  *   Dequantized weight: scale * (code - zero).
@@ -57,7 +65,7 @@ typedef enum {
 } dmr_status_t;
 
 typedef struct {
-    int32_t bits;       /* 4 or 8 */
+    int32_t bits;       /* 3, 4 or 8 */
     int32_t group_size; /* 64, 128, ... (multiple of 32, divides K), or 0 = one group per row */
 } dmr_qformat_t;
 
@@ -102,9 +110,9 @@ dmr_status_t dmr_dequantize(const void *qweight, const void *scales, const void 
                             int K, dmr_qformat_t f, void *W_out, dmr_out_t out, void *stream);
 
 /*
- * Low-precision linear layer (the W4A16 model's Linear, Sec. 5): Y = X . dequant(Wq)^T with fp32
- * accumulation.  Up to 32 rows run the bandwidth-bound decode kernels, larger M the tensor-core
- * kernels.  The decode kernels start fetching qweight, scales and zeros before the preceding kernel
+ * Low-precision linear layer (the W4A16 model's Linear, Sec. 5; also 8-bit and 3-bit codes): Y = X . dequant(Wq)^T
+ * with fp32 accumulation.  Up to 32 rows run the bandwidth-bound decode kernels, larger M the tensor-core
+ * kernels (3-bit codes: the decode kernel at every M, 16 rows per launch).  The decode kernels start fetching qweight, scales and zeros before the preceding kernel
  * of `stream` has finished (programmatic dependent launch): these three must be complete when the
  * call is enqueued, or be written by kernels that do not release their dependents early (dmr_quantize
  * and every ordinary kernel launch qualify).  X may be produced by the preceding kernel.
