@@ -257,3 +257,64 @@ def router_threshold(cal_scores, rho: float) -> float:
 def router_mask(scores, tau: float) -> np.ndarray:
     """mask[m] = 1 where the step's router score reaches the threshold (p_t >= tau: high precision), else 0."""
     return (np.asarray(scores).astype(np.float64) >= float(tau)).astype(np.uint8)
+
+
+def router_forward(Z, lengths, params, heads: int):
+    """Forward pass of the step-level router (Sec. 4.1 "Router Architecture"), in float64:
+
+        H_t = TransformerEnc_theta(X_t + P_t, m_t),   pi_theta(r_t | s_t) = Softmax(W h_t*),
+
+    X_t = [z_task, z_1, ..., z_t] (one row of Z per sequence, `lengths[b]` valid entries first: the valid-step mask m_t),
+    P_t learned positional embeddings, h_t* the encoder's output at the last valid step.
+
+    The paper fixes neither width, heads, feed-forward size, normalisation placement nor activation.  Reading taken: the
+    encoder layer of "Attention is all you need" - post-layer-norm, x <- LN(x + MHA(x)), x <- LN(x + W2 relu(W1 x + b1) + b2),
+    scaled dot-product attention over the valid steps only (padded steps are never keys; attention among valid steps is
+    not causal: the sequence already ends at the step being decided), LN with eps = 1e-5 over the feature axis, no dropout.
+
+    Z [B][L][d]; lengths [B] (1 <= len <= L); params: dict with
+      "pos" [L_max][d]; "layers": list of dicts with "wqkv" [3d][d] (rows: queries, keys, values), "bqkv" [3d], "wo" [d][d],
+      "bo" [d], "ln1_g", "ln1_b" [d], "w1" [f][d], "b1" [f], "w2" [d][f], "b2" [d], "ln2_g", "ln2_b" [d];
+      "wc" [C][d], "bc" [C].
+    Returns probabilities [B][C].
+    """
+    Z = np.asarray(Z, dtype=np.float64)
+    B, L, d = Z.shape
+    dh = d // heads
+    if dh * heads != d:
+        raise ValueError("heads must divide d")
+    pos = np.asarray(params["pos"], dtype=np.float64)
+    out = np.zeros((B, np.asarray(params["wc"]).shape[0]), dtype=np.float64)
+
+    def layer_norm(x, g, b):
+        mu = x.mean(axis=-1, keepdims=True)
+        var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+        return (x - mu) / np.sqrt(var + 1e-5) * g + b
+
+    for b in range(B):
+        n = int(lengths[b])
+        if not 1 <= n <= L:
+            raise ValueError("lengths must lie in [1, L]")
+        x = Z[b, :n, :] + pos[:n, :]                      # X_t + P_t, valid steps only
+        for lay in params["layers"]:
+            wqkv = np.asarray(lay["wqkv"], dtype=np.float64)
+            qkv = x @ wqkv.T + np.asarray(lay["bqkv"], dtype=np.float64)
+            q, k, v = qkv[:, :d], qkv[:, d:2 * d], qkv[:, 2 * d:]
+            att = np.zeros_like(x)
+            for h in range(heads):
+                sl = slice(h * dh, (h + 1) * dh)
+                s = (q[:, sl] @ k[:, sl].T) / np.sqrt(float(dh))
+                s = s - s.max(axis=-1, keepdims=True)
+                p = np.exp(s)
+                p = p / p.sum(axis=-1, keepdims=True)
+                att[:, sl] = p @ v[:, sl]
+            y = att @ np.asarray(lay["wo"], dtype=np.float64).T + np.asarray(lay["bo"], dtype=np.float64)
+            x = layer_norm(x + y, np.asarray(lay["ln1_g"], dtype=np.float64), np.asarray(lay["ln1_b"], dtype=np.float64))
+            hdn = np.maximum(x @ np.asarray(lay["w1"], dtype=np.float64).T + np.asarray(lay["b1"], dtype=np.float64), 0.0)
+            y = hdn @ np.asarray(lay["w2"], dtype=np.float64).T + np.asarray(lay["b2"], dtype=np.float64)
+            x = layer_norm(x + y, np.asarray(lay["ln2_g"], dtype=np.float64), np.asarray(lay["ln2_b"], dtype=np.float64))
+        hstar = x[n - 1]                                   # last-valid-step pooling
+        logits = np.asarray(params["wc"], dtype=np.float64) @ hstar + np.asarray(params["bc"], dtype=np.float64)
+        e = np.exp(logits - logits.max())
+        out[b] = e / e.sum()
+    return out

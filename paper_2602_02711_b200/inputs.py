@@ -151,3 +151,49 @@ def step_offsets(T: int, mean_len: int = 12, seed: int = 0, index: int = 0) -> n
     while offs[-1] < T:
         offs.append(min(T, offs[-1] + int(g.integers(0, 2 * mean_len + 1))))
     return np.asarray(offs, dtype=np.int32)
+
+
+# ---- the step-level router (Sec. 4.1): random-init parameters and synthetic step embeddings ----
+TID_ROUTER_PARAM = 81
+TID_ROUTER_EMB = 82
+TID_ROUTER_LEN = 83
+
+
+def router_params(d: int, heads: int, ffn: int, layers: int, l_max: int, classes: int, seed: int = 0) -> dict:
+    """Random-init parameters of the router's encoder as float32 arrays (the paper times its router with random weights
+    too, App. "Per-call router coefficient").  Matrices ~ N(0, 1/fan_in), biases and positional embeddings small,
+    layer-norm gains near one.  Shapes: see the oracle's router_forward."""
+    g = _rng(seed, TID_ROUTER_PARAM, d * 131 + layers)
+
+    def mat(rows, cols):
+        return (g.standard_normal((rows, cols)) / np.sqrt(cols)).astype(np.float32)
+
+    def vec(n, scale=0.05, base=0.0):
+        return (base + scale * g.standard_normal(n)).astype(np.float32)
+
+    del heads  # the head count does not change any shape
+    p = {"pos": (0.1 * g.standard_normal((l_max, d))).astype(np.float32), "layers": []}
+    for _ in range(layers):
+        p["layers"].append({
+            "wqkv": mat(3 * d, d), "bqkv": vec(3 * d), "wo": mat(d, d), "bo": vec(d),
+            "ln1_g": vec(d, 0.05, 1.0), "ln1_b": vec(d),
+            "w1": mat(ffn, d), "b1": vec(ffn), "w2": mat(d, ffn), "b2": vec(d),
+            "ln2_g": vec(d, 0.05, 1.0), "ln2_b": vec(d),
+        })
+    p["wc"] = mat(classes, d)
+    p["bc"] = vec(classes)
+    return p
+
+
+def router_embeddings(B: int, L: int, d: int, seed: int = 0, index: int = 0) -> np.ndarray:
+    """Z [B][L][d] float32: stand-ins for the frozen sentence encoder's step embeddings (unit-scale normal rows)."""
+    return _rng(seed, TID_ROUTER_EMB, index).standard_normal((B, L, d)).astype(np.float32)
+
+
+def router_lengths(B: int, L: int, seed: int = 0, index: int = 0) -> np.ndarray:
+    """Valid entries per sequence (task embedding + steps so far), uniform in [1, L]; the first and last sequence take
+    the extremes 1 and L."""
+    n = _rng(seed, TID_ROUTER_LEN, index).integers(1, L + 1, size=B, dtype=np.int64).astype(np.int32)
+    n[0] = 1
+    n[-1] = L
+    return n
