@@ -228,6 +228,35 @@ dmr_status_t dmr_router_calibrate(const float *cal_scores, int n, double rho, do
 dmr_status_t dmr_router_mask(const float *scores, int M, const double *tau, uint8_t *mask, void *stream);
 
 /*
+ * Forward pass of the step-level router (Sec. 4.1 "Router Architecture"): the sequence X_t = [z_task, z_1, ..., z_t] of
+ * task and step embeddings plus learned positional embeddings P_t goes through a masked Transformer encoder,
+ * H_t = TransformerEnc(X_t + P_t, m_t); the encoder's output at the last valid step, h_t*, gives the distribution over
+ * the precision choices, Softmax(W h_t*).  The paper fixes neither sizes, normalisation placement nor activation; the
+ * layer implemented is the original Transformer's encoder layer: x <- LN(x + MHA(x)), x <- LN(x + W2 relu(W1 x + b1) + b2),
+ * padded steps never attended to, no causal mask, LN eps 1e-5.  fp32 arithmetic.
+ *   cfg: d (model width: multiple of 16, 16..1024), heads (divides d), ffn (multiple of 16), layers (1..64),
+ *        l_max (positions, 1..128), classes (precision choices, 1..32).
+ *   params: device fp32, dmr_router_param_floats(cfg) values, 16-byte aligned, in this order:
+ *        pos [l_max][d];  per layer: wqkv [3d][d] (rows: queries, keys, values), bqkv [3d], wo [d][d], bo [d],
+ *        ln1_g [d], ln1_b [d], w1 [ffn][d], b1 [ffn], w2 [d][ffn], b2 [d], ln2_g [d], ln2_b [d];  wc [classes][d], bc [classes].
+ *   Z: device fp32 [B][L][d] (embeddings from the frozen encoder; L <= l_max; truncating a longer trajectory is the
+ *        caller's choice).  lengths: device int32 [B], valid entries per sequence, valid steps first, 1 <= lengths[b] <= L
+ *        (values outside are clamped into that range).  Entries of Z behind a sequence's length are ignored.
+ *   probs: device fp32 [B][classes].  scores: NULL, or device fp32 [B] that receives probs[b][score_class] - the
+ *        vector dmr_router_calibrate and dmr_router_mask take (score_class = the high-precision choice).
+ *   workspace: dmr_router_workspace_bytes(cfg, B, L) bytes, 16-byte aligned, no initial contents required.
+ * B = 0 is a no-op.  Errors: DMR_ERR_INVALID_ARG (sizes, NULL), DMR_ERR_ALIGNMENT, DMR_ERR_WORKSPACE.
+ */
+typedef struct {
+    int32_t d, heads, ffn, layers, l_max, classes;
+} dmr_router_cfg_t;
+size_t dmr_router_param_floats(dmr_router_cfg_t cfg);               /* 0 if cfg is invalid */
+size_t dmr_router_workspace_bytes(dmr_router_cfg_t cfg, int B, int L); /* 0 if cfg, B or L is invalid */
+dmr_status_t dmr_router_forward(const float *params, dmr_router_cfg_t cfg, const float *Z, const int32_t *lengths, int B,
+                                int L, float *probs, float *scores, int score_class, void *workspace,
+                                size_t workspace_bytes, void *stream);
+
+/*
  * Self-test of the bounded waits (no counterpart in the paper).  Every wait inside the kernels gives up after a
  * fixed number of polls, writes DMR_ERR_TIMEOUT to the workspace's status word and lets the kernel finish, so a
  * copy that never lands cannot hang the GPU.  This call launches one warp that waits - with the limit lowered

@@ -37,6 +37,12 @@ class QFormat(ctypes.Structure):
 _lib = None
 
 
+class RouterCfg(ctypes.Structure):
+    """dmr_router_cfg_t: sizes of the step-level router's encoder (Sec. 4.1)."""
+    _fields_ = [("d", ctypes.c_int32), ("heads", ctypes.c_int32), ("ffn", ctypes.c_int32), ("layers", ctypes.c_int32),
+                ("l_max", ctypes.c_int32), ("classes", ctypes.c_int32)]
+
+
 def lib_path() -> str:
     return _LIB_PATH
 
@@ -80,6 +86,12 @@ def lib() -> ctypes.CDLL:
     L.dmr_router_calibrate.argtypes = [vp, i32, ctypes.c_double, vp, vp]
     L.dmr_router_mask.restype = i32
     L.dmr_router_mask.argtypes = [vp, i32, vp, vp, vp]
+    L.dmr_router_param_floats.restype = sz
+    L.dmr_router_param_floats.argtypes = [RouterCfg]
+    L.dmr_router_workspace_bytes.restype = sz
+    L.dmr_router_workspace_bytes.argtypes = [RouterCfg, i32, i32]
+    L.dmr_router_forward.restype = i32
+    L.dmr_router_forward.argtypes = [vp, RouterCfg, vp, vp, i32, i32, vp, vp, i32, vp, sz, vp]
     L.dmr_selftest_wait_timeout.restype = i32
     L.dmr_selftest_wait_timeout.argtypes = [vp, sz, vp]
     L.dmr_workspace_status.restype = i32
@@ -326,3 +338,43 @@ def dmr_router_mask(scores: torch.Tensor, tau: torch.Tensor, stream=None) -> tor
     mask = torch.empty(scores.numel(), dtype=torch.uint8, device=scores.device)
     _check(lib().dmr_router_mask(_ptr(scores), scores.numel(), _ptr(tau), _ptr(mask), _stream(stream)))
     return mask
+
+
+def pack_router_params(params: dict, cfg: RouterCfg, device="cuda") -> torch.Tensor:
+    """Lays a dict of router parameters (numpy / torch arrays, shapes as in include/dmr.h) out as the one fp32 device
+    buffer dmr_router_forward reads: pos; per layer wqkv, bqkv, wo, bo, ln1_g, ln1_b, w1, b1, w2, b2, ln2_g, ln2_b; wc, bc."""
+    n = lib().dmr_router_param_floats(cfg)
+    if n == 0:
+        raise DmrError(1, "invalid router configuration")
+    parts = [params["pos"]]
+    for lay in params["layers"]:
+        parts += [lay[k] for k in ("wqkv", "bqkv", "wo", "bo", "ln1_g", "ln1_b", "w1", "b1", "w2", "b2", "ln2_g", "ln2_b")]
+    parts += [params["wc"], params["bc"]]
+    flat = torch.cat([torch.as_tensor(a, dtype=torch.float32).reshape(-1) for a in parts])
+    if flat.numel() != n or len(params["layers"]) != cfg.layers:
+        raise DmrError(1, "router parameters do not match the configuration")
+    return flat.to(device)
+
+
+def dmr_router_forward(params: torch.Tensor, cfg: RouterCfg, Z: torch.Tensor, lengths: torch.Tensor, score_class: int = 0,
+                       workspace=None, stream=None):
+    """Router forward on the device: Z [B][L][d] fp32, lengths [B] int32 -> (probs [B][classes], scores [B] =
+    probs[:, score_class]), both fp32 on the device."""
+    _dev(params, torch.float32, "params")
+    _dev(Z, torch.float32, "Z")
+    _dev(lengths, torch.int32, "lengths")
+    B, L, d = Z.shape
+    if d != cfg.d or lengths.numel() != B:
+        raise DmrError(1, "shape mismatch")
+    probs = torch.empty((B, cfg.classes), dtype=torch.float32, device=Z.device)
+    scores = torch.empty(B, dtype=torch.float32, device=Z.device)
+    if B == 0:
+        return probs, scores
+    need = lib().dmr_router_workspace_bytes(cfg, B, L)
+    if need == 0:
+        raise DmrError(1, "invalid router configuration or sizes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=Z.device)
+    _check(lib().dmr_router_forward(_ptr(params), cfg, _ptr(Z), _ptr(lengths), B, L, _ptr(probs), _ptr(scores), int(score_class),
+                                    _ptr(workspace), workspace.numel(), _stream(stream)))
+    return probs, scores

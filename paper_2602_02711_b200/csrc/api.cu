@@ -499,6 +499,38 @@ int dmr_describe_dispatch(dmr_op_t op, int M, int N, int K, dmr_qformat_t f, cha
                     (M + kStreamChunk - 1) / kStreamChunk);
 }
 
+static bool router_cfg_ok(const dmr_router_cfg_t &c) {
+    if (c.d < 16 || c.d > 1024 || c.d % 16 != 0) return false;
+    if (c.heads < 1 || c.d % c.heads != 0) return false;
+    if (c.ffn < 16 || c.ffn % 16 != 0 || c.ffn > 65536) return false;
+    if (c.layers < 1 || c.layers > 64) return false;
+    if (c.l_max < 1 || c.l_max > 128) return false;
+    if (c.classes < 1 || c.classes > 32) return false;
+    return router_attention_smem(c.l_max, c.d / c.heads) <= 200 * 1024;
+}
+
+size_t dmr_router_param_floats(dmr_router_cfg_t cfg) { return router_cfg_ok(cfg) ? router_param_floats(cfg) : 0; }
+
+size_t dmr_router_workspace_bytes(dmr_router_cfg_t cfg, int B, int L) {
+    if (!router_cfg_ok(cfg) || B < 1 || L < 1 || L > cfg.l_max) return 0;
+    return router_workspace_bytes(cfg, B, L);
+}
+
+dmr_status_t dmr_router_forward(const float *params, dmr_router_cfg_t cfg, const float *Z, const int32_t *lengths, int B,
+                                int L, float *probs, float *scores, int score_class, void *workspace,
+                                size_t workspace_bytes, void *stream) {
+    if (!router_cfg_ok(cfg) || B < 0 || L < 1 || L > cfg.l_max) return DMR_ERR_INVALID_ARG;
+    if ((long long)B * L > (1ll << 24)) return DMR_ERR_UNSUPPORTED;
+    if (scores && (score_class < 0 || score_class >= cfg.classes)) return DMR_ERR_INVALID_ARG;
+    if (B == 0) return DMR_OK;
+    if (!params || !Z || !lengths || !probs) return DMR_ERR_INVALID_ARG;
+    if (!aligned16(params) || !aligned16(Z)) return DMR_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < router_workspace_bytes(cfg, B, L)) return DMR_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return DMR_ERR_ALIGNMENT;
+    return launch_router_forward(params, cfg, Z, lengths, B, L, probs, scores, score_class, reinterpret_cast<float *>(workspace),
+                                 (cudaStream_t)stream);
+}
+
 dmr_status_t dmr_router_calibrate(const float *cal_scores, int n, double rho, double *tau, void *stream) {
     if (!cal_scores || !tau || n < 1) return DMR_ERR_INVALID_ARG;
     if (!(rho >= 0.0 && rho <= 1.0)) return DMR_ERR_INVALID_ARG;

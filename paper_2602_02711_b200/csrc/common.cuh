@@ -149,6 +149,13 @@ dmr_status_t launch_stepwise_kl(const void *high, const void *low, bool f32, int
 dmr_status_t launch_router_calibrate(const float *scores, int n, double rho, double *tau, double *picked, cudaStream_t st);
 dmr_status_t launch_router_mask(const float *scores, int M, const double *tau, uint8_t *mask, cudaStream_t st);
 
+// Router forward (Sec. 4.1): fp32 parameters in the layout dmr.h documents; ws holds router_workspace_bytes().
+size_t router_param_floats(const dmr_router_cfg_t &c);
+size_t router_workspace_bytes(const dmr_router_cfg_t &c, int B, int L);
+size_t router_attention_smem(int L, int dh);
+dmr_status_t launch_router_forward(const float *params, const dmr_router_cfg_t &c, const float *Z, const int32_t *lengths, int B,
+                                   int L, float *probs, float *scores, int score_class, float *ws, cudaStream_t st);
+
 // One warp waits on a barrier nobody arrives at, with a short limit: *status becomes DMR_ERR_TIMEOUT, *returned 2.
 dmr_status_t launch_wait_timeout_selftest(int32_t *status, int32_t *returned, cudaStream_t st);
 
