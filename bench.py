@@ -239,7 +239,7 @@ def run_ours(args):
     peaks = load_peaks()
     fmt = QFormat(BITS, GROUP)
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost", "w3", "kl", "crossover"}
+    sections = set(args.sections.split(",")) if args.sections else {"decode", "e2e", "cpu", "prefill", "routed", "dense", "quantize", "layer_cost", "w3", "router", "kl", "crossover"}
 
     def bf16_dev(bits_np):
         return torch.from_numpy(bits_np.view(np.int16)).view(torch.bfloat16).to(dev)
@@ -603,6 +603,37 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, l2_b
         out["w3_vs_w4_decode_7b"] = {k: {"t_w4_us": round(v["t_w4_us_per_layer"], 1), "t_w3_us": round(v["t_w3_us_per_layer"], 1),
                                          "ratio": round(v["t_w4_over_t_w3"], 3)} for k, v in w3.items()}
 
+    if "router" in sections:
+        # The step-level router's forward pass (Sec. 4.1) at the default depth of 8 layers on sentence-encoder-sized
+        # embeddings (width 384, 6 heads, feed-forward 1536, 2 precision choices; the paper prints none of these sizes),
+        # random-init weights as in the paper's own timing (App. "Per-call router coefficient"), sequences of 1 .. 32
+        # entries.  One call decides B concurrent agent steps.  fp32 CUDA-core arithmetic: the roofline is the fp32
+        # FMA peak, 148 SMs x 128 lanes x 2 flop x 1.965 GHz = 74.5 TFLOP/s.
+        from paper_2602_02711_b200 import RouterCfg
+        kw = dict(d=384, heads=6, ffn=1536, layers=8, l_max=32, classes=2)
+        cfg = RouterCfg(**kw)
+        params = dmr.pack_router_params(inputs.router_params(**kw, seed=0), cfg, dev)
+        L = 32
+        rt = {}
+        for B in (1, 64):
+            Z = torch.from_numpy(inputs.router_embeddings(B, L, kw["d"], seed=0)).to(dev)
+            n = torch.from_numpy(inputs.router_lengths(B, L, seed=0)).to(dev)
+            wsr = torch.empty(dmr.lib().dmr_router_workspace_bytes(cfg, B, L), dtype=torch.uint8, device=dev)
+            g = torch.cuda.CUDAGraph()
+            dmr.dmr_router_forward(params, cfg, Z, n, 1, workspace=wsr)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                dmr.dmr_router_forward(params, cfg, Z, n, 1, workspace=wsr)
+            t = timeit(g.replay, reps=20, warm=3)
+            T = B * L
+            flops = 2.0 * T * kw["layers"] * (4 * kw["d"] * kw["d"] + 2 * kw["d"] * kw["ffn"])
+            rt[f"B{B}"] = {"ms_per_call": t * 1e3, "tokens": T, "tflops_fp32": flops / t / 1e12,
+                           "frac_fp32_fma_peak": flops / t / 1e12 / 74.5, "launches_per_call": 2 + 7 * kw["layers"]}
+        rt["config"] = dict(kw, note="sizes are this build's reading; the paper prints none")
+        rt["paper_t_router_ms_per_call"] = "17.13-29.15 (A6000, router plus frozen sentence encoder)"
+        emit_section("router_forward", rt)
+        out["router_forward"] = {k: {"ms": round(v["ms_per_call"], 3), "frac_fp32": round(v["frac_fp32_fma_peak"], 3)} for k, v in rt.items() if k.startswith("B")}
+
     if "crossover" in sections:
         # 32B-class gate and down linears, INT4 g=64 and INT8 per-channel, M = 1 .. 256, 1 % outlier channels x20,
         # with the library's default dispatch (decode kernels up to 32 rows, tensor-core kernels above): where
@@ -673,7 +704,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost,w3,kl (default: all; none = headline only)")
+    ap.add_argument("--sections", default="", help="comma list: decode,e2e,cpu,prefill,routed,dense,quantize,crossover,layer_cost,w3,router,kl (default: all; none = headline only)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
