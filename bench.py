@@ -41,14 +41,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 def emit_section(name, obj):
-    """Full per-section results go out as a line of their own (and into gpurun_out/ when that folder exists); the
-    final line of the run only carries short summaries."""
+    """Full per-section results go out as a line of their own (and are appended to the file DMR_BENCH_SECTIONS names, if
+    set); the final line of the run only carries short summaries."""
     line = json.dumps({"section": name, "results": obj})
     print(line, flush=True)
-    d = os.path.join(ROOT, "gpurun_out")
-    if os.path.isdir(d):
+    path = os.environ.get("DMR_BENCH_SECTIONS")
+    if path:
         try:
-            with open(os.path.join(d, "bench_sections.jsonl"), "a") as f:
+            with open(path, "a") as f:
                 f.write(line + "\n")
         except OSError:
             pass
@@ -629,7 +629,7 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, l2_b
             flops = 2.0 * T * kw["layers"] * (4 * kw["d"] * kw["d"] + 2 * kw["d"] * kw["ffn"])
             rt[f"B{B}"] = {"ms_per_call": t * 1e3, "tokens": T, "tflops_fp32": flops / t / 1e12,
                            "frac_fp32_fma_peak": flops / t / 1e12 / 74.5, "launches_per_call": 2 + 7 * kw["layers"]}
-        rt["config"] = dict(kw, note="sizes are this build's reading; the paper prints none")
+        rt["config"] = dict(kw, note="sizes are this library's reading; the paper prints none")
         rt["paper_t_router_ms_per_call"] = "17.13-29.15 (A6000, router plus frozen sentence encoder)"
         emit_section("router_forward", rt)
         out["router_forward"] = {k: {"ms": round(v["ms_per_call"], 3), "frac_fp32": round(v["frac_fp32_fma_peak"], 3)} for k, v in rt.items() if k.startswith("B")}

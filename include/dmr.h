@@ -56,7 +56,7 @@ extern "C" {
 typedef enum {
     DMR_OK = 0,
     DMR_ERR_INVALID_ARG = 1, /* null pointer, negative size, K not a multiple of the group ... */
-    DMR_ERR_UNSUPPORTED = 2, /* a format or shape this build has no kernel for */
+    DMR_ERR_UNSUPPORTED = 2, /* a format or shape the library has no kernel for */
     DMR_ERR_ALIGNMENT = 3,   /* a pointer is not 16-byte aligned */
     DMR_ERR_WORKSPACE = 4,   /* workspace is NULL or smaller than dmr_workspace_bytes() */
     DMR_ERR_NONFINITE = 5,   /* written to dev_status by dmr_quantize: NaN/Inf weight seen */

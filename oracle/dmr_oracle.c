@@ -34,7 +34,7 @@
  *                                  3*(i%10)..+2 when i%10 < 5 and at bits 16+3*(i%10-5)..+2 otherwise (five codes in
  *                                  each half-word, bit 15 and bit 31 left over); bit b of code 30 is bit 15 of word b,
  *                                  bit b of code 31 is bit 31 of word b.  (The paper gives no 3-bit layout: its W3
- *                                  checkpoint is expanded to fp16 at load time.  This one is defined by this build.)
+ *                                  checkpoint is expanded to fp16 at load time.  This one is defined by this library.)
  *   scales  [N][K/g] bf16 bits,  zeros [N][K/g] uint8
  *   Y  [M][N] binary64
  */

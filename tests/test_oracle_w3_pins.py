@@ -1,6 +1,6 @@
 """Pins of the oracle's 3-bit format (the W3A16, group-128 variant of Sec. 5 / App. "Quantization Detail").
 
-The paper keeps its 3-bit checkpoint expanded to fp16 and prints no layout, so the layout is this build's: every 32 codes
+The paper keeps its 3-bit checkpoint expanded to fp16 and prints no layout, so the layout is this library's own: every 32 codes
 take three 32-bit words; code i < 30 of a block sits in word i // 10, five codes per half-word (bits 3j.. for j = i % 10 < 5,
 bits 16 + 3(j - 5).. otherwise); bit b of code 30 is bit 15 of word b, bit b of code 31 is bit 31 of word b.  The pins use an
 independent Python packer written from that sentence, a closed-form lossless group, the quantization rule in exact rational
