@@ -13,7 +13,7 @@
 // Arithmetic: fp32 throughout (CUDA cores; fused multiply-adds), so that the probabilities agree with a binary64
 // evaluation to about 1e-6 and the comparison against a threshold is stable.  The model is small (14 M parameters at
 // d = 384 and 8 layers) and runs once per agent step, next to a language-model call of tens of milliseconds.
-// Kernels: positions added; per layer a tiled linear (QKV), one CTA per (sequence, head) for the attention, a linear
+// Kernels: positions added; per layer a linear (QKV; tiled, or one feature per warp when there are at most 32 tokens), one CTA per (sequence, head) for the attention, a linear
 // with the residual added, a layer norm, two linears (ReLU; residual), a layer norm; then pooling, head and softmax.
 #include "sm100.cuh"
 
@@ -103,6 +103,53 @@ __global__ void __launch_bounds__(256) router_linear_kernel(const float *__restr
     }
 }
 
+// The same linear for at most 32 tokens (one agent deciding one step): a 64 x 64 tile per CTA would leave most SMs idle,
+// so a CTA takes two output features and all tokens, four warps per feature each with a quarter of the k range - the
+// weight row is read once, 16 bytes per lane, the activations come through the L1 - and the sums are reduced across
+// the warp and then across the four warps (in a fixed order) at the end.
+constexpr int kSmallT = 32;
+template <bool RELU, bool RESID>
+__global__ void __launch_bounds__(256) router_linear_small_kernel(const float *__restrict__ X, const float *__restrict__ W,
+                                                                  const float *__restrict__ bias, const float *__restrict__ R,
+                                                                  int T, int N, int K, float *__restrict__ Y) {
+    __shared__ float part[2][4][kSmallT];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int f = warp >> 2, ks = warp & 3;
+    const int n = blockIdx.x * 2 + f;
+    const int kq = K / 4;  // K is a multiple of 16
+    float acc[kSmallT];
+#pragma unroll
+    for (int t = 0; t < kSmallT; ++t) acc[t] = 0.f;
+    if (n < N) {
+        for (int k = ks * kq + 4 * lane; k < (ks + 1) * kq; k += 128) {
+            const float4 w = __ldg(reinterpret_cast<const float4 *>(W + (size_t)n * K + k));
+#pragma unroll
+            for (int t = 0; t < kSmallT; ++t) {
+                if (t < T) {
+                    const float4 x = __ldg(reinterpret_cast<const float4 *>(X + (size_t)t * K + k));
+                    acc[t] = fmaf(w.x, x.x, fmaf(w.y, x.y, fmaf(w.z, x.z, fmaf(w.w, x.w, acc[t]))));
+                }
+            }
+        }
+    }
+    float mine = 0.f;  // lane t keeps token t's sum
+#pragma unroll
+    for (int t = 0; t < kSmallT; ++t) {
+        float v = acc[t];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        if (lane == t) mine = v;
+    }
+    part[f][ks][lane] = mine;
+    __syncthreads();
+    if (ks == 0 && n < N && lane < T) {
+        float v = ((part[f][0][lane] + part[f][1][lane]) + part[f][2][lane]) + part[f][3][lane] + bias[n];
+        if (RELU) v = fmaxf(v, 0.f);
+        if (RESID) v += R[(size_t)lane * N + n];
+        Y[(size_t)lane * N + n] = v;
+    }
+}
+
 // One CTA per (sequence, head): softmax(Q K^T / sqrt(dh)) V over the valid steps.  QKV [T][3 d] (queries, keys, values),
 // O [T][d].  Keys and values of the head sit in shared memory (rows padded by one float); a warp takes query rows
 // warp, warp + 4, ...; every lane scores the keys lane, lane + 32, ... (L <= 128) and then sums its columns of V.
@@ -127,7 +174,10 @@ __global__ void __launch_bounds__(kAttWarps * 32) router_attention_kernel(const 
     }
     __syncthreads();
     const float scale = 1.0f / sqrtf((float)dh);
-    for (int l = warp; l < L; l += kAttWarps) {
+    // this CTA's share of the query rows (gridDim.z CTAs per sequence and head)
+    const int rows_per = (L + gridDim.z - 1) / gridDim.z;
+    const int l_lo = blockIdx.z * rows_per, l_hi = min(L, l_lo + rows_per);
+    for (int l = l_lo + warp; l < l_hi; l += kAttWarps) {
         float *orow = O + (row0 + l) * (size_t)d + h * dh;
         if (l >= n) {  // a padded step: nothing reads its row; keep it finite
             for (int c = lane; c < dh; c += 32) orow[c] = 0.f;
@@ -236,8 +286,12 @@ __global__ void __launch_bounds__(32) router_head_kernel(const float *__restrict
 template <bool RELU, bool RESID>
 dmr_status_t launch_linear(const float *X, const float *W, const float *bias, const float *R, int T, int N, int K, float *Y,
                            cudaStream_t st) {
-    dim3 grid((unsigned)((N + LBN - 1) / LBN), (unsigned)((T + LBM - 1) / LBM), 1);
-    router_linear_kernel<RELU, RESID><<<grid, 256, 0, st>>>(X, W, bias, R, T, N, K, Y);
+    if (T <= kSmallT) {
+        router_linear_small_kernel<RELU, RESID><<<(N + 1) / 2, 256, 0, st>>>(X, W, bias, R, T, N, K, Y);
+    } else {
+        dim3 grid((unsigned)((N + LBN - 1) / LBN), (unsigned)((T + LBM - 1) / LBM), 1);
+        router_linear_kernel<RELU, RESID><<<grid, 256, 0, st>>>(X, W, bias, R, T, N, K, Y);
+    }
     return check_launch();
 }
 
@@ -282,7 +336,10 @@ dmr_status_t launch_router_forward(const float *params, const dmr_router_cfg_t &
         const float *w2 = b1 + f, *b2 = w2 + (size_t)d * f, *ln2_g = b2 + d, *ln2_b = ln2_g + d;
         p = ln2_b + d;
         if ((r = launch_linear<false, false>(H, wqkv, bqkv, nullptr, T, 3 * d, d, QKV, st)) != DMR_OK) return r;
-        router_attention_kernel<<<dim3((unsigned)B, (unsigned)c.heads, 1), kAttWarps * 32, att_smem, st>>>(QKV, lengths, L, d, dh, ATT);
+        // few sequences: split a sequence's query rows over several CTAs (each loads the head's keys and values again)
+        int zsplit = (4 * 148) / (B * c.heads);
+        zsplit = zsplit < 1 ? 1 : (zsplit > (L + kAttWarps - 1) / kAttWarps ? (L + kAttWarps - 1) / kAttWarps : zsplit);
+        router_attention_kernel<<<dim3((unsigned)B, (unsigned)c.heads, (unsigned)zsplit), kAttWarps * 32, att_smem, st>>>(QKV, lengths, L, d, dh, ATT);
         if ((r = check_launch()) != DMR_OK) return r;
         if ((r = launch_linear<false, true>(ATT, wo, bo, H, T, d, d, SUM, st)) != DMR_OK) return r;
         router_layernorm_kernel<<<ln_blocks, 256, 0, st>>>(SUM, ln1_g, ln1_b, T, d, H);

@@ -43,6 +43,9 @@ def run(cfg_kw, B, L, seed, lengths=None):
     (dict(d=128, heads=1, ffn=64, layers=2, l_max=128, classes=1), 3, 128),       # one head of width 128, the longest sequence, one class
     (dict(d=1024, heads=16, ffn=1024, layers=1, l_max=8, classes=32), 2, 8),      # the widest model and the most classes
     (dict(d=48, heads=3, ffn=80, layers=16, l_max=5, classes=2), 9, 5),           # head width 16, deep
+    (dict(d=384, heads=6, ffn=1536, layers=8, l_max=32, classes=2), 1, 32),       # one agent, one decision: the 32-token instance of the linears
+    (dict(d=64, heads=4, ffn=128, layers=3, l_max=12, classes=3), 2, 8),          # 16 tokens
+    (dict(d=64, heads=4, ffn=128, layers=3, l_max=12, classes=3), 1, 1),          # a single token
 ])
 def test_router_forward_matches_oracle(cfg_kw, B, L):
     run(cfg_kw, B, L, seed=B + L)
