@@ -598,10 +598,27 @@ def run_extra_sections(sections, rank, dev, torch, dmr, inputs, fmt, peaks, l2_b
                            "w4_weight_gbs": layer_w4 / t4 / 1e9, "w3_weight_gbs": layer_w3 / t3 / 1e9,
                            "w3_frac_hbm": layer_w3 / t3 / 1e9 / peaks["hbm_gbs"],
                            "paper_projection_t_w4_over_t_w3": 1.15}
+        # prefill-sized batches: the same tensor-core kernel with the 3-bit unpack (codes read from global memory by the
+        # unpack threads) against the 4-bit one, four linears, M = 2048
+        t3p = t4p = flops = 0.0
+        for n, (N, K) in inputs.LAYER_7B.items():
+            Xp = randx(2048, K, 9)
+            Yp = torch.empty((2048, N), dtype=torch.bfloat16, device=dev)
+            for fq, Qs in ((f3, Q3s), (f4, Q4s)):
+                wsp = dmr.new_workspace(0, 2048, N, K, fq, dev)
+                t = timeit(lambda: dmr.dmr_lowbit_linear(Xp, Qs[0][n], OUT_BF16, Y=Yp, workspace=wsp), reps=10, warm=3)
+                if fq is f3:
+                    t3p += t
+                else:
+                    t4p += t
+            flops += 2.0 * 2048 * N * K
+        w3["prefill_M2048"] = {"t_w4_us": t4p * 1e6, "t_w3_us": t3p * 1e6, "w4_tflops": flops / t4p / 1e12, "w3_tflops": flops / t3p / 1e12,
+                               "w3_frac_bf16_burst": flops / t3p / 1e12 / peaks["bf16_tflops"]}
         del Q3s, Q4s
         emit_section("w3_vs_w4_decode_7b", w3)
         out["w3_vs_w4_decode_7b"] = {k: {"t_w4_us": round(v["t_w4_us_per_layer"], 1), "t_w3_us": round(v["t_w3_us_per_layer"], 1),
-                                         "ratio": round(v["t_w4_over_t_w3"], 3)} for k, v in w3.items()}
+                                         "ratio": round(v["t_w4_over_t_w3"], 3)} for k, v in w3.items() if k.startswith("M")}
+        out["w3_prefill_M2048_tflops"] = round(w3["prefill_M2048"]["w3_tflops"], 1)
 
     if "router" in sections:
         # The step-level router's forward pass (Sec. 4.1) at the default depth of 8 layers on sentence-encoder-sized

@@ -112,7 +112,7 @@ dmr_status_t dmr_dequantize(const void *qweight, const void *scales, const void 
 /*
  * Low-precision linear layer (the W4A16 model's Linear, Sec. 5; also 8-bit and 3-bit codes): Y = X . dequant(Wq)^T
  * with fp32 accumulation.  Up to 32 rows run the bandwidth-bound decode kernels, larger M the tensor-core
- * kernels (3-bit codes: the decode kernel at every M, 16 rows per launch).  The decode kernels start fetching qweight, scales and zeros before the preceding kernel
+ * kernels (3-bit codes: the persistent tensor-core kernel where it applies, otherwise the decode kernel, 16 rows per launch).  The decode kernels start fetching qweight, scales and zeros before the preceding kernel
  * of `stream` has finished (programmatic dependent launch): these three must be complete when the
  * call is enqueued, or be written by kernels that do not release their dependents early (dmr_quantize
  * and every ordinary kernel launch qualify).  X may be produced by the preceding kernel.

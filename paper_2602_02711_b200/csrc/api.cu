@@ -62,7 +62,13 @@ bool decode_w4_enabled() {
 
 constexpr int kDecodeChunk = 16;  // rows one launch of the 4-bit decode kernel takes at most
 
-bool use_gemm(int M, int N, int K, int bits, int g) { return M > decode_max_m() && gemm_supported(M, N, K, bits, g); }
+// Whether a call goes to the tensor-core kernels.  For 3-bit codes that family is the persistent prefill kernel alone
+// (no split-K kernel): batches it does not take stay on the decode kernel, 16 rows per launch.
+bool use_gemm(int M, int N, int K, int bits, int g) {
+    if (M <= decode_max_m()) return false;
+    if (bits == 3) return prefill_supported(M, N, K, bits, g);
+    return gemm_supported(M, N, K, bits, g);
+}
 
 Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f) {
     Scratch s;

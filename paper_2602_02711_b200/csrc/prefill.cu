@@ -1,4 +1,4 @@
-// Prefill-sized low-bit linear layers (M in the hundreds and above): a persistent, warp-specialised
+// Prefill-sized low-bit linear layers (M in the hundreds and above; 3-, 4- and 8-bit codes): a persistent, warp-specialised
 // tcgen05 GEMM with the dequantisation fused into the operand pipeline.  Prefill is a dense
 // contraction (its cost is folded into the per-token latency, App. "Latency coefficients"), so it
 // belongs on the tensor cores.
@@ -42,7 +42,8 @@ struct PrefillCfg {
     static constexpr int A_BYTES = PM * PK * 2;              // 16 KB of fp16 weights
     static constexpr int B_BYTES = BN * PK * 2;              // activations
     static constexpr int P_ROW = PK * BITS / 8;              // packed bytes per feature per stage
-    static constexpr int P_BYTES = PM * P_ROW;               // 4 or 8 KB
+    static constexpr int P_BYTES = BITS == 3 ? 0 : PM * P_ROW;  // 4 or 8 KB (3-bit rows are 24 bytes per stage, which no
+                                                                // TMA box can be: the unpack threads read them from global memory)
     static constexpr int STAGE = A_BYTES + B_BYTES + ((P_BYTES + 1023) / 1024) * 1024;
     static constexpr int S_RAW = (212 * 1024) / STAGE;
     static constexpr int S = S_RAW > 8 ? 8 : S_RAW;
@@ -54,6 +55,7 @@ struct PrefillCfg {
 struct PrefillArgs {
     const uint16_t *scales;
     const uint8_t *zeros;
+    const uint32_t *qweight3;  // 3-bit codes (read by the unpack threads; 4- and 8-bit codes come through the tensor map)
     const float *xscale;   // power of two each prepared activation row was divided by
     void *Y;
     const int32_t *idx;    // routed: output row of batch slot m (nullptr = identity)
@@ -207,7 +209,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                     mbar_expect_tx(full_bar(s), TX);
                     tma_load_2d(b_tile(s), &map_x, full_bar(s), kb * PK, m0);
-                    tma_load_2d(p_tile(s), &map_w, full_bar(s), kb * Cfg::P_ROW, n0);
+                    if constexpr (BITS != 3) tma_load_2d(p_tile(s), &map_w, full_bar(s), kb * Cfg::P_ROW, n0);
                 }
             }
         }
@@ -267,9 +269,23 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 sb = __ldg(sp + kb / kb_per_group);
                 zb = __ldg(zp + kb / kb_per_group);
             }
+            // 3-bit codes: this row's six words of the stage, read from global memory one stage of this group ahead
+            const uint32_t *wrow = a.qweight3 + (size_t)n * (size_t)(a.K / 32 * 3);
+            uint2 w3a = make_uint2(0u, 0u), w3b = w3a, w3c = w3a;
+            if (BITS == 3 && kb < nkb) {
+                w3a = __ldg(reinterpret_cast<const uint2 *>(wrow + kb * 6));
+                w3b = __ldg(reinterpret_cast<const uint2 *>(wrow + kb * 6 + 2));
+                w3c = __ldg(reinterpret_cast<const uint2 *>(wrow + kb * 6 + 4));
+            }
             for (; kb < nkb; kb += NG) {
                 const uint32_t it = it0 + (uint32_t)kb;
                 const int s = it % S;
+                uint2 n3a = w3a, n3b = w3b, n3c = w3c;
+                if (BITS == 3 && kb + NG < nkb) {
+                    n3a = __ldg(reinterpret_cast<const uint2 *>(wrow + (kb + NG) * 6));
+                    n3b = __ldg(reinterpret_cast<const uint2 *>(wrow + (kb + NG) * 6 + 2));
+                    n3c = __ldg(reinterpret_cast<const uint2 *>(wrow + (kb + NG) * 6 + 4));
+                }
                 // scale / zero of this group's next k block, fetched while this block is unpacked
                 uint32_t sb_next = sb, zb_next = zb;
                 if (kb + NG < nkb) {
@@ -283,7 +299,53 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
                 const uint32_t src = p_tile(s) + r * Cfg::P_ROW;
                 const uint32_t dst = a_tile(s) + r * 128;
-                if (BITS == 4) {
+                if (BITS == 3) {
+                    // fp16 patterns: a half-word holds five codes at bits 0, 3, 6, 9, 12.  0x6400 | (bits 0..2) = 1024 + q,
+                    // 0x6400 | (bits 3..5) = 1024 + 8 q, 0x6400 | (bits 6..8) = 1024 + 64 q without a shift (10 mantissa
+                    // bits); one shift by 9 brings the last two down.  Minus the matching 1024 + zero is exact, then one
+                    // rounding of the product with s', s'/8 or s'/64.
+                    const float sf = __uint_as_float(sb << 16) * fdown;
+                    uint32_t s2, s2_8, s2_64;
+                    asm("cvt.rn.f16x2.f32 %0, %1, %1;" : "=r"(s2) : "f"(sf));
+                    asm("cvt.rn.f16x2.f32 %0, %1, %1;" : "=r"(s2_8) : "f"(sf * 0.125f));
+                    asm("cvt.rn.f16x2.f32 %0, %1, %1;" : "=r"(s2_64) : "f"(sf * 0.015625f));
+                    const uint32_t z1 = 0x6400u | zb, z8 = 0x6400u | (zb << 3), z64 = 0x6400u | (zb << 6);
+                    const uint32_t zo1 = z1 | (z1 << 16), zo8 = z8 | (z8 << 16), zo64 = z64 | (z64 << 16);
+                    const uint32_t words[6] = {w3a.x, w3a.y, w3b.x, w3b.y, w3c.x, w3c.y};
+#pragma unroll
+                    for (int blk = 0; blk < 2; ++blk) {  // 32 codes = three words = four 16-byte chunks of fp16 weights
+                        uint32_t D[16];  // pair 5 j + i = codes (10 j + i, 10 j + 5 + i); pair 15 = codes (30, 31)
+#pragma unroll
+                        for (int j = 0; j < 3; ++j) {
+                            const uint32_t u = words[3 * blk + j], u9 = u >> 9;
+                            D[5 * j + 0] = f16x2_mul(f16x2_sub(lop3_and_or(u, 0x00070007u, 0x64006400u), zo1), s2);
+                            D[5 * j + 1] = f16x2_mul(f16x2_sub(lop3_and_or(u, 0x00380038u, 0x64006400u), zo8), s2_8);
+                            D[5 * j + 2] = f16x2_mul(f16x2_sub(lop3_and_or(u, 0x01C001C0u, 0x64006400u), zo64), s2_64);
+                            D[5 * j + 3] = f16x2_mul(f16x2_sub(lop3_and_or(u9, 0x00070007u, 0x64006400u), zo1), s2);
+                            D[5 * j + 4] = f16x2_mul(f16x2_sub(lop3_and_or(u9, 0x00380038u, 0x64006400u), zo8), s2_8);
+                        }
+                        {
+                            uint32_t t = lop3_and_or(words[3 * blk] >> 15, 0x00010001u, 0x64006400u);
+                            t = lop3_and_or(words[3 * blk + 1] >> 14, 0x00020002u, t);
+                            t = lop3_and_or(words[3 * blk + 2] >> 13, 0x00040004u, t);
+                            D[15] = f16x2_mul(f16x2_sub(t, zo1), s2);
+                        }
+                        // code a of the block: pair and half it sits in; the tile wants neighbours (2 v, 2 v + 1) side by side
+                        auto pair_of = [](int a) { return a >= 30 ? 15 : 5 * (a / 10) + (a % 10) % 5; };
+                        auto high_of = [](int a) { return a >= 30 ? a - 30 : ((a % 10) >= 5 ? 1 : 0); };
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int v4 = 0; v4 < 4; ++v4) {
+                                const int a0 = 8 * c4 + 2 * v4, a1 = a0 + 1;
+                                o[v4] = prmt(D[pair_of(a0)], D[pair_of(a1)], (high_of(a1) ? 0x7600u : 0x5400u) | (high_of(a0) ? 0x32u : 0x10u));
+                            }
+                            const uint32_t addr = dst + ((((uint32_t)(4 * blk + c4)) ^ swz) << 4);
+                            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                        }
+                    }
+                } else if (BITS == 4) {
                     uint32_t w[CH];
 #pragma unroll
                     for (int c4 = 0; c4 < CH; c4 += 4)
@@ -339,6 +401,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (lane == 0) mbar_arrive(ready_bar(s));
                 sb = sb_next;
                 zb = zb_next;
+                w3a = n3a;
+                w3b = n3b;
+                w3c = n3c;
             }
         }
     } else {
@@ -438,7 +503,7 @@ int prefill_bn(int M, int N, int sms) {
 }  // namespace
 
 bool prefill_supported(int M, int N, int K, int bits, int g) {
-    if (!((bits == 4 || bits == 8) && K % PK == 0 && g % PK == 0 && K <= 32768)) return false;
+    if (!((bits == 3 || bits == 4 || bits == 8) && K % PK == 0 && g % PK == 0 && K <= 32768)) return false;
     if (M > 128) return true;
     // one tile of rows: only when the feature tiles alone fill most of the SMs (no split-K here; the
     // split-K kernel takes the layers with few output features)
@@ -476,12 +541,16 @@ dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qw
                             (uint32_t)bn, PK, TmaSwizzle::k128B))
         return DMR_ERR_CUDA;
     const uint64_t row_bytes = (uint64_t)K * bits / 8;
-    if (!make_tensor_map_2d(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qweight, (uint64_t)N, row_bytes, row_bytes, PM,
-                            (uint32_t)(PK * bits / 8), TmaSwizzle::kNone))
+    if (bits == 3) {
+        map_w = map_x;  // not used: a stage of 3-bit codes is 24 bytes per row, the unpack threads load it themselves
+    } else if (!make_tensor_map_2d(&map_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qweight, (uint64_t)N, row_bytes, row_bytes, PM,
+                                   (uint32_t)(PK * bits / 8), TmaSwizzle::kNone)) {
         return DMR_ERR_CUDA;
+    }
     PrefillArgs a;
     a.scales = scales;
     a.zeros = zeros;
+    a.qweight3 = reinterpret_cast<const uint32_t *>(qweight);
     a.xscale = xscale;
     a.Y = Y;
     a.idx = sel.idx;
@@ -495,6 +564,7 @@ dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qw
     a.m_tiles = (M + bn - 1) / bn;
     const long long tiles = (long long)a.n_tiles * a.m_tiles;
     const int grid = (int)(tiles < sms ? tiles : sms);
+    if (bits == 3) return bn == 256 ? launch_prefill_t<3, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<3, 128>(map_w, map_x, a, grid, out, st);
     if (bits == 4) return bn == 256 ? launch_prefill_t<4, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<4, 128>(map_w, map_x, a, grid, out, st);
     return bn == 256 ? launch_prefill_t<8, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<8, 128>(map_w, map_x, a, grid, out, st);
 }

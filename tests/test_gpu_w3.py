@@ -195,3 +195,55 @@ def test_w3_sizes_and_errors():
     W = to_dev_bf16(inputs.weights(4, 128, seed=0))
     with pytest.raises(dmr.DmrError):
         dmr.dmr_quantize(W, QFormat(3, 48))                          # groups hold whole blocks of 32 codes
+
+
+TOL_PREFILL = 3e-4  # the tensor-core kernel rounds each dequantized weight once to fp16's 11 significant bits
+
+
+@pytest.mark.parametrize("M,N,K,group", [
+    (300, 640, 512, 128),     # three row tiles of 128 / 256, five feature tiles
+    (150, 520, 1024, 128),    # ragged N and M
+    (257, 256, 384, 64),      # groups of 64 = one stage, M just over a row tile
+    (200, 128, 2048, 0),      # one group per row
+])
+def test_lowbit_linear_w3_prefill(M, N, K, group):
+    info = dmr.dmr_describe_dispatch(OP_LOWBIT, M, N, K, QFormat(3, group))
+    assert info["kernel"] == "prefill" and info["bits"] == 3
+    W = inputs.weights(N, K, seed=11, index=N + K)
+    X = inputs.activations(M, K, seed=11, index=M)
+    q, ref = quantize_both(W, group)
+    assert_quant_equal(q, ref)
+    Xd = to_dev_bf16(X)
+    Y32 = dmr.dmr_lowbit_linear(Xd, q, OUT_F32)
+    Yref = oracle.lowbit_linear(X, *ref, bits=3, group=group)
+    assert rel_err(Y32.cpu().numpy().astype(np.float64), Yref) <= TOL_PREFILL
+    assert torch.equal(dmr.dmr_lowbit_linear(Xd, q, OUT_BF16), Y32.to(torch.bfloat16))
+
+
+def test_w3_prefill_outliers_and_routed_rows():
+    M, N, K = 200, 384, 1024
+    W = inputs.weights(N, K, seed=12)
+    X = inputs.activations(M, K, seed=12, outlier_frac=0.01)
+    mask = inputs.precision_mask(M, p_high=0.3, seed=12)
+    q, ref = quantize_both(W, 128)
+    Wd, Xd = to_dev_bf16(W), to_dev_bf16(X)
+    Yl = dmr.dmr_lowbit_linear(Xd, q, OUT_F32)
+    assert rel_err(Yl.cpu().numpy().astype(np.float64), oracle.lowbit_linear(X, *ref, bits=3, group=128)) <= TOL_PREFILL
+    Y = dmr.dmr_routed_linear(Xd, torch.from_numpy(mask).cuda(), Wd, q, OUT_F32)
+    Yh = dmr.dmr_dense_linear(Xd, Wd, OUT_F32)
+    for m in range(M):
+        assert torch.equal(Y[m], Yh[m] if mask[m] else Yl[m])
+
+
+def test_w3_prefill_7b_layer_sampled():
+    N, K, M = 4096, 4096, 2048
+    W = inputs.weights(N, K, seed=13)
+    X = inputs.activations(M, K, seed=13)
+    q = dmr.dmr_quantize(to_dev_bf16(W), QFormat(3, 128))
+    ref = oracle.quantize(W, bits=3, group=128)
+    assert_quant_equal(q, ref)
+    Y = dmr.dmr_lowbit_linear(to_dev_bf16(X), q, OUT_F32).cpu().numpy().astype(np.float64)
+    ms, ns = inputs.sample_outputs(M, N, 4096, seed=13)
+    want = oracle.sampled_linear(X, ms, ns, qweight=ref[0], scales=ref[1], zeros=ref[2], bits=3, group=128)
+    assert float(np.abs(Y[ms, ns] - want).max() / np.abs(want).max()) <= TOL_PREFILL
+    assert np.isfinite(Y).all()
