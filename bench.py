@@ -402,6 +402,13 @@ def run_ours(args):
             summary["prefill_M8192"] = {"tflops": round(rp["achieved"], 1), "us": round(rp["us"], 1)}
         if "routed" in result:
             summary["routed_14b_M64"] = {"layer_us": round(result["routed"]["layer_us"], 1), "frac_hbm": round(result["routed"]["frac_hbm"], 3)}
+        if "w3_vs_w4_decode_7b" in result:
+            w = result.pop("w3_vs_w4_decode_7b")
+            summary["t_w4_over_t_w3"] = {k: v["ratio"] for k, v in w.items()}
+            if "w3_prefill_M2048_tflops" in result:
+                summary["w3_prefill_M2048_tflops"] = result.pop("w3_prefill_M2048_tflops")
+        if "router_forward" in result:
+            summary["router_forward_ms"] = {k: v["ms"] for k, v in result.pop("router_forward").items()}
         for key in ("crossover_32b", "dense_decode_frac_hbm", "layer_cost_7b", "stepwise_kl"):
             if key in result:
                 summary[key] = result.pop(key)
