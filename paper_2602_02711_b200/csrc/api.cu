@@ -98,7 +98,7 @@ Scratch carve(void *workspace, dmr_op_t op, int M, int N, int K, dmr_qformat_t f
         s.prefill_scratch = base + off;
         off += round_up(prefill_scratch_bytes(M, K), 256);
     }
-    const size_t partial_low = low_gemm ? gemm_plan(M, N, K, f.bits).partial_bytes : 0;
+    const size_t partial_low = !low_gemm ? 0 : (prefill_supported(M, N, K, f.bits, g) ? prefill_partial_bytes(M, N, K) : gemm_plan(M, N, K, f.bits).partial_bytes);
     const size_t partial_dense = dense_gemm ? gemm_plan(M, N, K, 0).partial_bytes : 0;
     if (op == DMR_OP_ROUTED_LINEAR) {
         if (partial_low) {
@@ -149,7 +149,7 @@ dmr_status_t run_lowbit(const uint16_t *X, int M, RowSel sel, const uint32_t *qw
     const size_t ysz = out == DMR_OUT_F32 ? 4 : 2;
     if (use_gemm(M, N, K, f.bits, g)) {
         if (prefill_supported(M, N, K, f.bits, g))  // gathers the listed rows itself
-            return launch_prefill(X, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.prefill_scratch, ws.status, st);
+            return launch_prefill(X, M, sel, qweight, scales, zeros, N, K, f.bits, g, Y, out, ws.prefill_scratch, ws.partial, ws.status, st);
         const uint16_t *Xin = X;
         if (sel.idx) {
             dmr_status_t r = launch_gather_rows(X, K, M, sel.idx, sel.count, 0, ws.xg_low, st);
@@ -478,10 +478,10 @@ int dmr_describe_dispatch(dmr_op_t op, int M, int N, int K, dmr_qformat_t f, cha
     const int bits = dense ? 0 : f.bits, g = dense ? K : group_of(K, f);
     if (use_gemm(M, N, K, bits, g)) {
         if (!dense && prefill_supported(M, N, K, bits, g)) {
-            int bn, ctas;
+            int bn, splits, ctas;
             long long tiles;
-            prefill_plan(M, N, &bn, &tiles, &ctas);
-            return snprintf(buf, buf_bytes, "prefill bits=%d bn=%d tiles=%lld ctas=%d", bits, bn, tiles, ctas);
+            prefill_plan(M, N, K, &bn, &splits, &tiles, &ctas);
+            return snprintf(buf, buf_bytes, "prefill bits=%d bn=%d splits=%d tiles=%lld ctas=%d", bits, bn, splits, tiles, ctas);
         }
         const GemmPlan p = gemm_plan(M, N, K, bits);
         return snprintf(buf, buf_bytes, "gemm bits=%d bn=%d splits=%d", bits, p.bn, p.splits);

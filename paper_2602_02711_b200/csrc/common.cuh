@@ -98,17 +98,19 @@ dmr_status_t launch_decode_w3(const uint16_t *X, int M, RowSel sel, const uint32
 void decode_w4_plan(int M, int g, int *nt, int *r, int *warps);
 void decode_w3_plan(int M, int *nt, int *r, int *warps);
 void stream_plan(int M, int N, int K, int bits, int *tiles, long long *steps, int *cluster);
-void prefill_plan(int M, int N, int *bn, long long *tiles, int *ctas);
+void prefill_plan(int M, int N, int K, int *bn, int *splits, long long *tiles, int *ctas);
 
 // Persistent prefill GEMM (M > 32, low-bit weights); sel.idx maps batch slots to rows of X and Y, sel.count
 // says how many slots are valid.
 bool prefill_supported(int M, int N, int K, int bits, int g);
 // X is the caller's activation matrix (for a routed call the rows sel.idx lists are gathered);
-// `scratch` holds prefill_scratch_bytes(M, K) bytes for the prepared fp16 activations and their row scales.
+// `scratch` holds prefill_scratch_bytes(M, K) bytes for the prepared fp16 activations and their row scales, `partial`
+// prefill_partial_bytes(M, N, K) bytes of fp32 partial sums (0 unless the call is split along k).
 size_t prefill_scratch_bytes(int M, int K);
+size_t prefill_partial_bytes(int M, int N, int K);
 dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qweight, const uint16_t *scales,
                             const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
-                            void *scratch, int32_t *status, cudaStream_t st);
+                            void *scratch, float *partial, int32_t *status, cudaStream_t st);
 
 // Tensor-core GEMM family (M > 16): tcgen05 MMA with TMA-staged operands.
 struct GemmPlan {
@@ -124,6 +126,9 @@ GemmPlan gemm_plan(int M, int N, int K, int bits);
 dmr_status_t launch_gemm(const uint16_t *X, int M, RowSel sel, const void *weights, const uint16_t *scales,
                          const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
                          float *partial, int32_t *status, cudaStream_t st);
+// Y[row(m)][n] = sum over z < splits of partial[z][m][n], in split order (fp32 partial sums by batch slot).
+dmr_status_t launch_splitk_reduce(const float *partial, int splits, int M, int N, RowSel sel, void *Y, dmr_out_t out,
+                                  cudaStream_t st);
 // Xg[s] = X[idx[s]] for the list slots coff <= coff + s < *count (s < Mcap); other slots are zero-filled.
 // `idx` is already advanced to slot coff.
 dmr_status_t launch_gather_rows(const uint16_t *X, int K, int Mcap, const int32_t *idx, const int32_t *count,

@@ -443,6 +443,18 @@ dmr_status_t launch_gemm(const uint16_t *X, int M, RowSel sel, const void *weigh
     return r;
 }
 
+dmr_status_t launch_splitk_reduce(const float *partial, int splits, int M, int N, RowSel sel, void *Y, dmr_out_t out,
+                                  cudaStream_t st) {
+    const size_t total = (size_t)M * N;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (out == DMR_OUT_F32)
+        splitk_reduce_kernel<true><<<blocks, 256, 0, st>>>(partial, splits, M, N, sel.idx, sel.count, Y);
+    else
+        splitk_reduce_kernel<false><<<blocks, 256, 0, st>>>(partial, splits, M, N, sel.idx, sel.count, Y);
+    return check_launch();
+}
+
 dmr_status_t launch_gather_rows(const uint16_t *X, int K, int Mcap, const int32_t *idx, const int32_t *count,
                                 int coff, uint16_t *Xg, cudaStream_t st) {
     const size_t total = (size_t)Mcap * (K / 8);

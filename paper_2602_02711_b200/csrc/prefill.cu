@@ -63,6 +63,11 @@ struct PrefillArgs {
     int32_t *status;
     int M, N, K, g_size;
     int n_tiles, m_tiles;
+    // split-K (batches of one row tile on layers with few feature tiles): a work item is (tile, split); split z sums the
+    // k blocks [z kb_per_split, (z + 1) kb_per_split) and writes fp32 partial sums [z][M][N] that a second kernel adds
+    // up in split order.  splits == 1: the tile's whole k range, outputs written directly.
+    float *partial;
+    int splits, kb_per_split;
 };
 
 
@@ -189,7 +194,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const int nkb = a.K / PK;
     // a routed call sizes the grid for M rows but only the first `rows` slots hold anything
     const int rows = a.count ? min(*a.count, a.M) : a.M;
-    const int total_tiles = a.n_tiles * ((rows + BN - 1) / BN);
+    const int total_tiles = a.n_tiles * ((rows + BN - 1) / BN) * a.splits;  // work items: (tile, split), split fastest
     const int G = a.K / a.g_size;
     const int kb_per_group = a.g_size / PK;  // >= 1
 
@@ -200,8 +205,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             uint32_t it = 0;  // k blocks issued so far, over all tiles
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int n0 = (tile % a.n_tiles) * PM, m0 = (tile / a.n_tiles) * BN;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const int split = tile % a.splits, tl = tile / a.splits;
+                const int kb_lo = split * a.kb_per_split, kb_hi = min(nkb, kb_lo + a.kb_per_split);
+                const int n0 = (tl % a.n_tiles) * PM, m0 = (tl / a.n_tiles) * BN;
+                for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
                     const int s = it % S;
                     if (it >= (uint32_t)S && !mbar_wait(empty_bar(s), ((it / S) - 1) & 1, a.status)) {
                         ok = false;
@@ -225,7 +232,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (tile_it >= 2 && !mbar_wait(tempty_bar(buf), ((tile_it >> 1) - 1) & 1, a.status)) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const int kb_lo = (tile % a.splits) * a.kb_per_split, kb_hi = min(nkb, kb_lo + a.kb_per_split);
+                for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
                     const int s = it % S;
                     if (!mbar_wait(ready_bar(s), (it / S) & 1, a.status)) {
                         ok = false;
@@ -235,7 +243,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < PK / 16; ++j)
                         umma_bf16_ss(d_tmem, umma_desc_sw128(a_tile(s) + j * 32), umma_desc_sw128(b_tile(s) + j * 32), IDESC,
-                                     (kb == 0 && j == 0) ? 0u : 1u);
+                                     (kb == kb_lo && j == 0) ? 0u : 1u);
                     umma_commit(empty_bar(s));
                 }
                 if (ok) umma_commit(tfull_bar(buf));
@@ -251,10 +259,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         constexpr int CH = 8, c_lo = 0;               // 16-byte chunks (8 weights each) per thread and stage
         const int grp_id = (warp - 2) >> 2;
         const uint32_t swz = (uint32_t)(r & 7);
-        uint32_t it0 = 0;  // running number of the tile's first stage
+        uint32_t it0 = 0;  // running number of the work item's first stage
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, it0 += (uint32_t)nkb) {
-            const int n = min((tile % a.n_tiles) * PM + r, a.N - 1);
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            const int split = tile % a.splits, tl = tile / a.splits;
+            const int kb_lo = split * a.kb_per_split, kb_hi = min(nkb, kb_lo + a.kb_per_split);
+            const int n = min((tl % a.n_tiles) * PM + r, a.N - 1);
             const uint16_t *sp = a.scales + (size_t)n * G;
             const uint8_t *zp = a.zeros + (size_t)n * G;
             // power of two of the feature's largest scale: s' = s * 2^-f lies in (0, 2)
@@ -263,32 +273,32 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             int fb = (int)(smax >> 7);
             fb = fb < 1 ? 1 : (fb > 253 ? 253 : fb);
             const float fdown = __uint_as_float((uint32_t)(254 - fb) << 23);  // 2^-(fb - 127)
-            int kb = (int)(((uint32_t)grp_id + (uint32_t)NG - it0 % (uint32_t)NG) % (uint32_t)NG);  // this group's first k block of the tile
+            int kb = kb_lo + (int)(((uint32_t)grp_id + (uint32_t)NG - it0 % (uint32_t)NG) % (uint32_t)NG);  // this group's first k block of the item
             uint32_t sb = 0, zb = 0;
-            if (kb < nkb) {
+            if (kb < kb_hi) {
                 sb = __ldg(sp + kb / kb_per_group);
                 zb = __ldg(zp + kb / kb_per_group);
             }
             // 3-bit codes: this row's six words of the stage, read from global memory one stage of this group ahead
             const uint32_t *wrow = a.qweight3 + (size_t)n * (size_t)(a.K / 32 * 3);
             uint2 w3a = make_uint2(0u, 0u), w3b = w3a, w3c = w3a;
-            if (BITS == 3 && kb < nkb) {
+            if (BITS == 3 && kb < kb_hi) {
                 w3a = __ldg(reinterpret_cast<const uint2 *>(wrow + kb * 6));
                 w3b = __ldg(reinterpret_cast<const uint2 *>(wrow + kb * 6 + 2));
                 w3c = __ldg(reinterpret_cast<const uint2 *>(wrow + kb * 6 + 4));
             }
-            for (; kb < nkb; kb += NG) {
-                const uint32_t it = it0 + (uint32_t)kb;
+            for (; kb < kb_hi; kb += NG) {
+                const uint32_t it = it0 + (uint32_t)(kb - kb_lo);
                 const int s = it % S;
                 uint2 n3a = w3a, n3b = w3b, n3c = w3c;
-                if (BITS == 3 && kb + NG < nkb) {
+                if (BITS == 3 && kb + NG < kb_hi) {
                     n3a = __ldg(reinterpret_cast<const uint2 *>(wrow + (kb + NG) * 6));
                     n3b = __ldg(reinterpret_cast<const uint2 *>(wrow + (kb + NG) * 6 + 2));
                     n3c = __ldg(reinterpret_cast<const uint2 *>(wrow + (kb + NG) * 6 + 4));
                 }
                 // scale / zero of this group's next k block, fetched while this block is unpacked
                 uint32_t sb_next = sb, zb_next = zb;
-                if (kb + NG < nkb) {
+                if (kb + NG < kb_hi) {
                     const int grp = (kb + NG) / kb_per_group;
                     sb_next = __ldg(sp + grp);
                     zb_next = __ldg(zp + grp);
@@ -405,6 +415,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 w3b = n3b;
                 w3c = n3c;
             }
+            it0 += (uint32_t)(kb_hi - kb_lo);
         }
     } else {
         // ================= epilogue warps =================
@@ -414,7 +425,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         uint32_t tile_it = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
             const int buf = tile_it & 1;
-            const int n = (tile % a.n_tiles) * PM + r, m0 = (tile / a.n_tiles) * BN;
+            const int split = tile % a.splits, tl = tile / a.splits;
+            const int n = (tl % a.n_tiles) * PM + r, m0 = (tl / a.n_tiles) * BN;
             // the power of two the unpack threads divided this feature's scales by, undone here
             uint32_t smax = 0;
             {
@@ -442,8 +454,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     for (int c = 0; c < 32; ++c) {
                         const int m = m0 + c0 + c;
                         if (m < rows) {
-                            const int row = a.idx ? a.idx[m] : m;
                             const float v = (__uint_as_float(u[c]) * __ldg(a.xscale + m)) * fscale;
+                            if (a.partial) {  // split-K: this split's share, by batch slot; the reduction scatters the rows
+                                a.partial[((size_t)split * a.M + m) * a.N + n] = v;
+                                continue;
+                            }
+                            const int row = a.idx ? a.idx[m] : m;
                             if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
                             else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
                         }
@@ -504,26 +520,52 @@ int prefill_bn(int M, int N, int sms) {
 
 bool prefill_supported(int M, int N, int K, int bits, int g) {
     if (!((bits == 3 || bits == 4 || bits == 8) && K % PK == 0 && g % PK == 0 && K <= 32768)) return false;
-    if (M > 128) return true;
-    // one tile of rows: only when the feature tiles alone fill most of the SMs (no split-K here; the
-    // split-K kernel takes the layers with few output features)
-    return M > 32 && (N + PM - 1) / PM >= 100;
+    if (M > 128 || bits == 3) return M > 32;  // 3-bit codes have no other tensor-core kernel
+    // one tile of rows: layers with at least 16 feature tiles (split along k when the tiles alone leave SMs idle); the
+    // narrow ones (k and v projections) are faster on the split-K kernel with the exact-integer operand
+    return M > 32 && (N + PM - 1) / PM >= 16;
 }
 
-void prefill_plan(int M, int N, int *bn, long long *tiles, int *ctas) {
+// Split-K factor: only for a single row tile (M <= 128) on layers whose feature tiles leave SMs idle.  As many splits
+// as give every SM at most one work item, each with at least sixteen k blocks.  Depends on (M, N, K) only.
+static int prefill_splits(int M, int N, int K, int sms, int *kb_per_split) {
+    const int nkb = K / PK, tiles = (N + PM - 1) / PM;
+    int splits = 1;
+    if (M <= 128 && tiles < sms) {
+        splits = sms / tiles;
+        if (splits > nkb / 16) splits = nkb / 16;  // a work item pays for its set-up (the feature's scale range) once
+        if (splits < 1) splits = 1;
+    }
+    *kb_per_split = (nkb + splits - 1) / splits;
+    return (nkb + *kb_per_split - 1) / *kb_per_split;  // no empty split
+}
+
+size_t prefill_partial_bytes(int M, int N, int K) {
+    int kbps;
+    const int splits = prefill_splits(M, N, K, prefill_sm_count(), &kbps);
+    return splits > 1 ? (size_t)splits * M * N * sizeof(float) : 0;
+}
+
+void prefill_plan(int M, int N, int K, int *bn, int *splits, long long *tiles, int *ctas) {
     const int sms = prefill_sm_count();
+    int kbps;
     *bn = prefill_bn(M, N, sms);
+    *splits = prefill_splits(M, N, K, sms, &kbps);
     *tiles = (long long)((N + PM - 1) / PM) * ((M + *bn - 1) / *bn);
-    *ctas = (int)(*tiles < sms ? *tiles : sms);
+    const long long items = *tiles * *splits;
+    *ctas = (int)(items < sms ? items : sms);
 }
 
 size_t prefill_scratch_bytes(int M, int K) { return round_up((size_t)M * K * 2, 256) + round_up((size_t)M * 4, 256); }
 
 dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qweight, const uint16_t *scales,
                             const uint8_t *zeros, int N, int K, int bits, int g, void *Y, dmr_out_t out,
-                            void *scratch, int32_t *status, cudaStream_t st) {
+                            void *scratch, float *partial, int32_t *status, cudaStream_t st) {
     const int sms = prefill_sm_count();
     const int bn = prefill_bn(M, N, sms);
+    int kb_per_split;
+    const int splits = prefill_splits(M, N, K, sms, &kb_per_split);
+    if (splits > 1 && !partial) return DMR_ERR_WORKSPACE;
     // activations: gather (routed calls), rescale each row by a power of two and convert to fp16
     uint16_t *Xh = reinterpret_cast<uint16_t *>(scratch);
     float *xscale = reinterpret_cast<float *>(reinterpret_cast<char *>(scratch) + round_up((size_t)M * K * 2, 256));
@@ -562,11 +604,17 @@ dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qw
     a.g_size = g;
     a.n_tiles = (N + PM - 1) / PM;
     a.m_tiles = (M + bn - 1) / bn;
-    const long long tiles = (long long)a.n_tiles * a.m_tiles;
+    a.splits = splits;
+    a.kb_per_split = kb_per_split;
+    a.partial = splits > 1 ? partial : nullptr;
+    const long long tiles = (long long)a.n_tiles * a.m_tiles * splits;
     const int grid = (int)(tiles < sms ? tiles : sms);
-    if (bits == 3) return bn == 256 ? launch_prefill_t<3, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<3, 128>(map_w, map_x, a, grid, out, st);
-    if (bits == 4) return bn == 256 ? launch_prefill_t<4, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<4, 128>(map_w, map_x, a, grid, out, st);
-    return bn == 256 ? launch_prefill_t<8, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<8, 128>(map_w, map_x, a, grid, out, st);
+    dmr_status_t r;
+    if (bits == 3) r = bn == 256 ? launch_prefill_t<3, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<3, 128>(map_w, map_x, a, grid, out, st);
+    else if (bits == 4) r = bn == 256 ? launch_prefill_t<4, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<4, 128>(map_w, map_x, a, grid, out, st);
+    else r = bn == 256 ? launch_prefill_t<8, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<8, 128>(map_w, map_x, a, grid, out, st);
+    if (r != DMR_OK || splits == 1) return r;
+    return launch_splitk_reduce(partial, splits, M, N, sel, Y, out, st);
 }
 
 }  // namespace dmr

@@ -119,7 +119,7 @@ def run_case(M, N, K, group, seed=0, outlier=0.0):
     (16, 4736, 1792, 128),   # several tiles per CTA
     (4, 256, 1024, 256),     # groups of two chunks
     (3, 96, 768, 0),         # one group per row
-    (40, 384, 512, 128),     # more rows than one launch takes: chunks of 16
+    (29, 384, 512, 128),     # more rows than one launch takes: chunks of 16
 ])
 def test_lowbit_linear_w3_decode(M, N, K, group):
     info = dmr.dmr_describe_dispatch(OP_LOWBIT, M, N, K, QFormat(3, group))
