@@ -146,7 +146,9 @@ xprep_kernel(const uint16_t *__restrict__ X, int K, int Mcap, const int32_t *__r
     }
 }
 
-template <int BITS, int BN, bool OUT_F32>
+// SPLITK: work items are (tile, split) and the epilogue writes fp32 partial sums; otherwise an item is a tile with its whole
+// k range (a compile-time choice: the large-batch instance carries none of the split bookkeeping).
+template <int BITS, int BN, bool OUT_F32, bool SPLITK>
 __global__ void __launch_bounds__(PrefillCfg<BITS, BN>::THREADS, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const PrefillArgs a) {
     using Cfg = PrefillCfg<BITS, BN>;
@@ -194,7 +196,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const int nkb = a.K / PK;
     // a routed call sizes the grid for M rows but only the first `rows` slots hold anything
     const int rows = a.count ? min(*a.count, a.M) : a.M;
-    const int total_tiles = a.n_tiles * ((rows + BN - 1) / BN) * a.splits;  // work items: (tile, split), split fastest
+    const int n_splits = SPLITK ? a.splits : 1;
+    const int total_tiles = a.n_tiles * ((rows + BN - 1) / BN) * n_splits;  // work items: (tile, split), split fastest
     const int G = a.K / a.g_size;
     const int kb_per_group = a.g_size / PK;  // >= 1
 
@@ -205,8 +208,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             uint32_t it = 0;  // k blocks issued so far, over all tiles
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int split = tile % a.splits, tl = tile / a.splits;
-                const int kb_lo = split * a.kb_per_split, kb_hi = min(nkb, kb_lo + a.kb_per_split);
+                const int split = SPLITK ? tile % n_splits : 0, tl = SPLITK ? tile / n_splits : tile;
+                const int kb_lo = SPLITK ? split * a.kb_per_split : 0, kb_hi = SPLITK ? min(nkb, kb_lo + a.kb_per_split) : nkb;
                 const int n0 = (tl % a.n_tiles) * PM, m0 = (tl / a.n_tiles) * BN;
                 for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
                     const int s = it % S;
@@ -232,7 +235,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (tile_it >= 2 && !mbar_wait(tempty_bar(buf), ((tile_it >> 1) - 1) & 1, a.status)) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                const int kb_lo = (tile % a.splits) * a.kb_per_split, kb_hi = min(nkb, kb_lo + a.kb_per_split);
+                const int kb_lo = SPLITK ? (tile % n_splits) * a.kb_per_split : 0, kb_hi = SPLITK ? min(nkb, kb_lo + a.kb_per_split) : nkb;
                 for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
                     const int s = it % S;
                     if (!mbar_wait(ready_bar(s), (it / S) & 1, a.status)) {
@@ -262,8 +265,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         uint32_t it0 = 0;  // running number of the work item's first stage
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-            const int split = tile % a.splits, tl = tile / a.splits;
-            const int kb_lo = split * a.kb_per_split, kb_hi = min(nkb, kb_lo + a.kb_per_split);
+            const int split = SPLITK ? tile % n_splits : 0, tl = SPLITK ? tile / n_splits : tile;
+            const int kb_lo = SPLITK ? split * a.kb_per_split : 0, kb_hi = SPLITK ? min(nkb, kb_lo + a.kb_per_split) : nkb;
             const int n = min((tl % a.n_tiles) * PM + r, a.N - 1);
             const uint16_t *sp = a.scales + (size_t)n * G;
             const uint8_t *zp = a.zeros + (size_t)n * G;
@@ -425,7 +428,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         uint32_t tile_it = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tile_it) {
             const int buf = tile_it & 1;
-            const int split = tile % a.splits, tl = tile / a.splits;
+            const int split = SPLITK ? tile % n_splits : 0, tl = SPLITK ? tile / n_splits : tile;
             const int n = (tl % a.n_tiles) * PM + r, m0 = (tl / a.n_tiles) * BN;
             // the power of two the unpack threads divided this feature's scales by, undone here
             uint32_t smax = 0;
@@ -455,7 +458,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         const int m = m0 + c0 + c;
                         if (m < rows) {
                             const float v = (__uint_as_float(u[c]) * __ldg(a.xscale + m)) * fscale;
-                            if (a.partial) {  // split-K: this split's share, by batch slot; the reduction scatters the rows
+                            if constexpr (SPLITK) {  // this split's share, by batch slot; the reduction scatters the rows
                                 a.partial[((size_t)split * a.M + m) * a.N + n] = v;
                                 continue;
                             }
@@ -487,8 +490,9 @@ dmr_status_t launch_prefill_t(const CUtensorMap &map_w, const CUtensorMap &map_x
         kernel<<<grid, Cfg::THREADS, Cfg::SMEM, st>>>(map_w, map_x, a);
         return check_launch();
     };
-    if (out == DMR_OUT_F32) return launch(prefill_kernel<BITS, BN, true>);
-    return launch(prefill_kernel<BITS, BN, false>);
+    if (a.splits > 1) return launch(prefill_kernel<BITS, BN, true, true>);  // partial sums are fp32 whatever the output
+    if (out == DMR_OUT_F32) return launch(prefill_kernel<BITS, BN, true, false>);
+    return launch(prefill_kernel<BITS, BN, false, false>);
 }
 
 int prefill_sm_count() {
