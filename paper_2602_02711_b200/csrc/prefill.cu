@@ -9,12 +9,12 @@
 // Per 64-wide k block and stage of the ring:
 //   warp 0      TMA: the packed code tile [128 features x 32 or 64 bytes] and the activation tile
 //               [BN rows x 128 bytes, 128-byte swizzle] land in shared memory (one mbarrier);
-//   warps 2..9  two threads per feature row turn its codes into the fp16 weights s' * (q - zero)
+//   warps 2..9 (2..13 for the 128-row tile)  one thread per feature row turns its codes into the fp16 weights s' * (q - zero)
 //               (exact integer q - zero, then ONE rounding of the product to 11 significant bits)
 //               and stores them as the swizzled K-major A tile;
 //   warp 1      one lane issues four tcgen05.mma (128 x BN x 16) that accumulate into one of two
 //               fp32 accumulators in tensor memory, and commits the stage back to the producer;
-//   warps 10..13 drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
+//   the last four warps drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
 //               next tile's MMAs run into the other accumulator.
 // CTAs are persistent: CTA b takes tiles b, b + grid, ...  Every wait is bounded.
 //
@@ -35,7 +35,6 @@ namespace {
 
 constexpr int PM = 128;  // features per tile (MMA M)
 constexpr int PK = 64;   // k per stage
-constexpr int UW = 8;    // unpack warps: UW / 4 groups of four, group i takes every (UW / 4)-th stage of the ring
 
 template <int BITS, int BN>
 struct PrefillCfg {
@@ -48,6 +47,9 @@ struct PrefillCfg {
     static constexpr int S_RAW = (212 * 1024) / STAGE;
     static constexpr int S = S_RAW > 8 ? 8 : S_RAW;
     static constexpr int TMEM_COLS = 2 * BN;                 // two accumulators
+    // unpack warps: UW / 4 groups of four, group i takes every (UW / 4)-th stage of the ring.  Three groups for the
+    // 128-row tile (small batches: a stage's MMAs are short and the unpack chain's latency is what is left), two for 256.
+    static constexpr int UW = BN == 128 ? 12 : 8;
     static constexpr int THREADS = 32 * (2 + UW + 4);
     static constexpr size_t SMEM = (size_t)S * STAGE + 1024 /*alignment*/ + 512 /*barriers*/;
 };
@@ -252,13 +254,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (ok) umma_commit(tfull_bar(buf));
             }
         }
-    } else if (warp < 2 + UW) {
+    } else if (warp < 2 + Cfg::UW) {
         // ================= unpack warps: codes -> fp16 weights s' * (q - zero) =================
         // A stage's chain (wait, load, convert, store, fence, arrive) is a string of shared-memory round trips that
         // one group of four warps cannot overlap with itself, so NG groups work on different stages of the ring
         // at the same time: group i takes the stages whose running number is i modulo NG.
         const int r = ((warp - 2) & 3) * 32 + lane;  // feature row of the tile
-        constexpr int NG = UW / 4;
+        constexpr int NG = Cfg::UW / 4;
         constexpr int CH = 8, c_lo = 0;               // 16-byte chunks (8 weights each) per thread and stage
         const int grp_id = (warp - 2) >> 2;
         const uint32_t swz = (uint32_t)(r & 7);
