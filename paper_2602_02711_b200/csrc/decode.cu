@@ -381,6 +381,9 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                             }
                         }
                 }
+                // the chunk whose activations are fetched during this one (after the CTA's last chunk the warp's first
+                // chunk once more: always a valid address)
+                const int next_chunk = sub == nsub - 1 ? (box + WARPS < nboxes ? box + WARPS : warp) * CPB : chunk + 1;
                 float gs[R][NT][4], sx[NT][4];
                 const uint32_t sxaddr = sxbase + (uint32_t)(((bl * CPB + sub) * NT) * 256 + lane * 8);
                 if constexpr (FAST) {
@@ -499,6 +502,14 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                     for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) b[nt][q] = xfrag4(nt, j, q);
+                        {   // the registers of this piece are free: fetch the same piece of the chunk to come now, a
+                            // chunk's worth of arithmetic ahead of its use (a miss in the L1 costs half a microsecond)
+                            const uint4 v = ldg_v4(xrow[nt] + next_chunk * CHUNK_K + 8 * j);
+                            x[nt][j][0] = v.x;
+                            x[nt][j][1] = v.y;
+                            x[nt][j][2] = v.z;
+                            x[nt][j][3] = v.w;
+                        }
                         if constexpr (!FAST) {
                             if (j == 0) mma_bf16_16816_zero(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
                             else mma_bf16_16816(sx[nt], kOnes, kOnes, kOnes, kOnes, b[nt][0], b[nt][1]);
@@ -533,9 +544,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) decode_w4_kernel(const __grid_c
                     }
                 }
                 }  // 4-bit codes
-                // the next chunk's activations
-                // (after the CTA's last chunk this reads the warp's first chunk once more: always a valid address)
-                load_x(sub == nsub - 1 ? (box + WARPS < nboxes ? box + WARPS : warp) * CPB : chunk + 1);
+                if constexpr (BITS == 3) load_x(next_chunk);  // (the 4-bit loop fetches piece by piece as it goes)
                 // the chunk lies inside one quantization group: s (sum x (128 + q) - (128 + z) sum x)
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
