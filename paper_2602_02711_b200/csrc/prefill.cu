@@ -54,6 +54,28 @@ struct PrefillCfg {
     static constexpr size_t SMEM = (size_t)S * STAGE + 1024 /*alignment*/ + 512 /*barriers*/;
 };
 
+// Largest magnitude pattern among a feature's G bf16 scales (sign bit cleared): eight scales per 16-byte load when the
+// row of the table allows it, so that a work item's set-up is a handful of independent loads, not a chain of G.
+__device__ __forceinline__ uint32_t scale_row_max(const uint16_t *sp, int G) {
+    uint32_t smax = 0;
+    if ((G & 7) == 0 && (reinterpret_cast<uintptr_t>(sp) & 15) == 0) {
+        uint32_t m0 = 0, m1 = 0;
+        for (int gi = 0; gi < G; gi += 8) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(sp + gi));
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                m0 = max(m0, w[i] & 0x7FFFu);
+                m1 = max(m1, (w[i] >> 16) & 0x7FFFu);
+            }
+        }
+        smax = max(m0, m1);
+    } else {
+        for (int gi = 0; gi < G; ++gi) smax = max(smax, (uint32_t)__ldg(sp + gi) & 0x7FFFu);
+    }
+    return smax;
+}
+
 struct PrefillArgs {
     const uint16_t *scales;
     const uint8_t *zeros;
@@ -273,8 +295,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const uint16_t *sp = a.scales + (size_t)n * G;
             const uint8_t *zp = a.zeros + (size_t)n * G;
             // power of two of the feature's largest scale: s' = s * 2^-f lies in (0, 2)
-            uint32_t smax = 0;
-            for (int gi = 0; gi < G; ++gi) smax = max(smax, (uint32_t)__ldg(sp + gi) & 0x7FFFu);
+            const uint32_t smax = scale_row_max(sp, G);
             int fb = (int)(smax >> 7);
             fb = fb < 1 ? 1 : (fb > 253 ? 253 : fb);
             const float fdown = __uint_as_float((uint32_t)(254 - fb) << 23);  // 2^-(fb - 127)
@@ -433,11 +454,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const int split = SPLITK ? tile % n_splits : 0, tl = SPLITK ? tile / n_splits : tile;
             const int n = (tl % a.n_tiles) * PM + r, m0 = (tl / a.n_tiles) * BN;
             // the power of two the unpack threads divided this feature's scales by, undone here
-            uint32_t smax = 0;
-            {
-                const uint16_t *sp = a.scales + (size_t)min(n, a.N - 1) * G;
-                for (int gi = 0; gi < G; ++gi) smax = max(smax, (uint32_t)__ldg(sp + gi) & 0x7FFFu);
-            }
+            const uint32_t smax = scale_row_max(a.scales + (size_t)min(n, a.N - 1) * G, G);
             int fb = (int)(smax >> 7);
             fb = fb < 1 ? 1 : (fb > 253 ? 253 : fb);
             const float fscale = __uint_as_float((uint32_t)fb << 23);  // 2^(fb - 127)
