@@ -381,12 +381,21 @@ GemmPlan gemm_plan(int M, int N, int K, int bits) {
     if (bits == 0 && M > 128) p.bn = 256;
     const int tiles = ((N + BM - 1) / BM) * ((M + p.bn - 1) / p.bn);
     const int kb = K / BK;
+    // Split-K factor: the one with the shortest longest path - waves of CTAs (one CTA per SM at a time) times the k blocks
+    // of a split plus a fixed cost per wave; at most 8 splits, at least 8 k blocks each.  (Rounding 148 / tiles up, as an
+    // earlier version did, put 160 CTAs on 148 SMs for 40 tiles: a second wave for twelve of them.)
     int splits = 1;
     if (tiles < 148) {
-        splits = (148 + tiles - 1) / tiles;
-        const int max_splits = kb / 8 > 0 ? kb / 8 : 1;
-        if (splits > max_splits) splits = max_splits;
-        if (splits > 8) splits = 8;
+        const int max_splits = kb / 8 > 0 ? (kb / 8 < 8 ? kb / 8 : 8) : 1;
+        long long best = -1;
+        for (int sp = 1; sp <= max_splits; ++sp) {
+            const long long waves = ((long long)tiles * sp + 147) / 148;
+            const long long cost = waves * ((kb + sp - 1) / sp + 4);
+            if (best < 0 || cost < best) {
+                best = cost;
+                splits = sp;
+            }
+        }
     }
     p.kblocks_per_split = (kb + splits - 1) / splits;
     p.splits = (kb + p.kblocks_per_split - 1) / p.kblocks_per_split;
