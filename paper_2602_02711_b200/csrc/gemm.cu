@@ -109,6 +109,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
 
+    // Set-up done: only now wait for the kernels before this one (gathered rows, row lists), and let the kernel behind
+    // this one start its own set-up.
+    pdl_wait();
+    pdl_launch_dependents();
     // quantization groups seen by this CTA: group boundaries in units of k-blocks
     const int kb_per_group = LOWBIT ? max(1, args.g_size / BK) : kb_total;
 
@@ -311,6 +315,8 @@ template <bool OUT_F32>
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float *__restrict__ partial, int splits, int M, int N, const int32_t *__restrict__ idx,
                      const int32_t *__restrict__ count, void *__restrict__ Y) {
+    pdl_wait();  // the partial sums come from the kernel before this one
+    pdl_launch_dependents();
     const int rows = count ? min(*count, M) : M;
     const size_t total = (size_t)rows * N;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
@@ -328,6 +334,8 @@ splitk_reduce_kernel(const float *__restrict__ partial, int splits, int M, int N
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const uint16_t *__restrict__ X, int K, int Mcap, const int32_t *__restrict__ idx,
                    const int32_t *__restrict__ count, int coff, uint16_t *__restrict__ Xg) {
+    pdl_wait();  // the row list comes from the kernel before this one
+    pdl_launch_dependents();
     const int rows = min(*count - coff, Mcap);
     const int vec_per_row = K / 8;
     const size_t total = (size_t)Mcap * vec_per_row;
@@ -346,7 +354,12 @@ dmr_status_t launch_gemm_t(const CUtensorMap &map_w, const CUtensorMap &map_x, c
     dim3 grid((a.N + BM - 1) / BM, (a.M + BN - 1) / BN, splits);
     auto launch = [&](auto kernel) -> dmr_status_t {
         if (!ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), Cfg::SMEM)) return DMR_ERR_CUDA;
-        kernel<<<grid, Cfg::THREADS, Cfg::SMEM, st>>>(map_w, map_x, a);
+        cudaError_t e = launch_pdl(kernel, grid, dim3(Cfg::THREADS), Cfg::SMEM, st, map_w, map_x, a);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            (void)cudaGetLastError();
+            return DMR_ERR_CUDA;
+        }
         return check_launch();
     };
     if (out == DMR_OUT_F32) return launch(gemm_kernel<MODE, BN, true>);
@@ -444,9 +457,9 @@ dmr_status_t launch_gemm(const uint16_t *X, int M, RowSel sel, const void *weigh
         int blocks = (int)((total + 255) / 256);
         if (blocks > 148 * 8) blocks = 148 * 8;
         if (out == DMR_OUT_F32)
-            splitk_reduce_kernel<true><<<blocks, 256, 0, st>>>(partial, p.splits, M, N, sel.idx, sel.count, Y);
+            (void)launch_pdl(splitk_reduce_kernel<true>, dim3((unsigned)blocks), dim3(256), 0, st, partial, p.splits, M, N, sel.idx, sel.count, Y);
         else
-            splitk_reduce_kernel<false><<<blocks, 256, 0, st>>>(partial, p.splits, M, N, sel.idx, sel.count, Y);
+            (void)launch_pdl(splitk_reduce_kernel<false>, dim3((unsigned)blocks), dim3(256), 0, st, partial, p.splits, M, N, sel.idx, sel.count, Y);
         r = check_launch();
     }
     return r;
@@ -458,9 +471,9 @@ dmr_status_t launch_splitk_reduce(const float *partial, int splits, int M, int N
     int blocks = (int)((total + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
     if (out == DMR_OUT_F32)
-        splitk_reduce_kernel<true><<<blocks, 256, 0, st>>>(partial, splits, M, N, sel.idx, sel.count, Y);
+        (void)launch_pdl(splitk_reduce_kernel<true>, dim3((unsigned)blocks), dim3(256), 0, st, partial, splits, M, N, sel.idx, sel.count, Y);
     else
-        splitk_reduce_kernel<false><<<blocks, 256, 0, st>>>(partial, splits, M, N, sel.idx, sel.count, Y);
+        (void)launch_pdl(splitk_reduce_kernel<false>, dim3((unsigned)blocks), dim3(256), 0, st, partial, splits, M, N, sel.idx, sel.count, Y);
     return check_launch();
 }
 
@@ -469,7 +482,7 @@ dmr_status_t launch_gather_rows(const uint16_t *X, int K, int Mcap, const int32_
     const size_t total = (size_t)Mcap * (K / 8);
     int blocks = (int)((total + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
-    gather_rows_kernel<<<blocks, 256, 0, st>>>(X, K, Mcap, idx, count, coff, Xg);
+    (void)launch_pdl(gather_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, st, X, K, Mcap, idx, count, coff, Xg);
     return check_launch();
 }
 

@@ -128,6 +128,8 @@ __global__ void __launch_bounds__(256)
 xprep_kernel(const uint16_t *__restrict__ X, int K, int Mcap, const int32_t *__restrict__ idx,
              const int32_t *__restrict__ count, uint16_t *__restrict__ Xh, float *__restrict__ xscale) {
     __shared__ uint32_t warp_max[8];
+    pdl_wait();               // nothing of the stream's earlier work is read or overwritten before this
+    pdl_launch_dependents();  // the GEMM behind this kernel may set itself up meanwhile
     const int rows = count ? min(*count, Mcap) : Mcap;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nv = K / 8;
@@ -217,6 +219,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
 
+    // Set-up done (barriers, tensor memory): only now wait for the kernels before this one - the prepared activations, the
+    // routed row lists - and let the kernel behind this one (the split-K sum) start its own set-up.
+    pdl_wait();
+    if constexpr (SPLITK) pdl_launch_dependents();  // (a large batch's successor would only sit on the SMs and wait)
     const int nkb = a.K / PK;
     // a routed call sizes the grid for M rows but only the first `rows` slots hold anything
     const int rows = a.count ? min(*a.count, a.M) : a.M;
@@ -506,7 +512,12 @@ dmr_status_t launch_prefill_t(const CUtensorMap &map_w, const CUtensorMap &map_x
     using Cfg = PrefillCfg<BITS, BN>;
     auto launch = [&](auto kernel) -> dmr_status_t {
         if (!ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), Cfg::SMEM)) return DMR_ERR_CUDA;
-        kernel<<<grid, Cfg::THREADS, Cfg::SMEM, st>>>(map_w, map_x, a);
+        cudaError_t e = launch_pdl(kernel, dim3((unsigned)grid), dim3(Cfg::THREADS), Cfg::SMEM, st, map_w, map_x, a);
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            (void)cudaGetLastError();
+            return DMR_ERR_CUDA;
+        }
         return check_launch();
     };
     if (a.splits > 1) return launch(prefill_kernel<BITS, BN, true, true>);  // partial sums are fp32 whatever the output
@@ -594,10 +605,16 @@ dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qw
     float *xscale = reinterpret_cast<float *>(reinterpret_cast<char *>(scratch) + round_up((size_t)M * K * 2, 256));
     {
         const int blocks = M < sms * 16 ? M : sms * 16;
-        if (K <= 2 * 2048) xprep_kernel<2><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
-        else if (K <= 8 * 2048) xprep_kernel<8><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
-        else if (K <= 16 * 2048) xprep_kernel<16><<<blocks, 256, 0, st>>>(X, K, M, sel.idx, sel.count, Xh, xscale);
+        cudaError_t e;
+        if (K <= 2 * 2048) e = launch_pdl(xprep_kernel<2>, dim3((unsigned)blocks), dim3(256), 0, st, X, K, M, sel.idx, sel.count, Xh, xscale);
+        else if (K <= 8 * 2048) e = launch_pdl(xprep_kernel<8>, dim3((unsigned)blocks), dim3(256), 0, st, X, K, M, sel.idx, sel.count, Xh, xscale);
+        else if (K <= 16 * 2048) e = launch_pdl(xprep_kernel<16>, dim3((unsigned)blocks), dim3(256), 0, st, X, K, M, sel.idx, sel.count, Xh, xscale);
         else return DMR_ERR_UNSUPPORTED;
+        if (e != cudaSuccess) {
+            g_last_cuda_error = (int)e;
+            (void)cudaGetLastError();
+            return DMR_ERR_CUDA;
+        }
         dmr_status_t r = check_launch();
         if (r != DMR_OK) return r;
     }

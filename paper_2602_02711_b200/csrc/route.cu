@@ -2,7 +2,7 @@
 // 1 = the step needs the high-precision weights (Sec. 4.2, "KL-to-Classification Mapping").
 // A stable partition turns it into two ascending row lists, so that each precision's rows can be
 // multiplied as one dense batch and written back at their own positions (step order).
-#include "common.cuh"
+#include "sm100.cuh"
 
 namespace dmr {
 
@@ -17,6 +17,8 @@ route_partition_kernel(const uint8_t *__restrict__ mask, int M, int32_t *__restr
     __shared__ int warp_high[32];
     __shared__ int base_high_s, base_low_s;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_wait();  // the lists may still be read, and the mask written, by kernels before this one
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         base_high_s = 0;
         base_low_s = 0;
@@ -60,7 +62,7 @@ route_partition_kernel(const uint8_t *__restrict__ mask, int M, int32_t *__restr
 
 dmr_status_t launch_route_partition(const uint8_t *mask, int M, int32_t *idx_high, int32_t *idx_low,
                                     int32_t *counts, cudaStream_t st) {
-    route_partition_kernel<<<1, kPartThreads, 0, st>>>(mask, M, idx_high, idx_low, counts);
+    (void)launch_pdl(route_partition_kernel, dim3(1), dim3(kPartThreads), 0, st, mask, M, idx_high, idx_low, counts);
     return check_launch();
 }
 

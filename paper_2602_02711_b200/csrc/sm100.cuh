@@ -257,6 +257,25 @@ __device__ __forceinline__ void mma_bf16_16816_zero(float (&d)[4], uint32_t a0, 
 }
 // Programmatic dependent launch: let the next kernel of the stream start; wait for the previous one
 // (all of its memory operations) before touching anything it may have written.
+// Host side: launches `kernel` so that it may start before the kernel before it in the stream has finished (programmatic
+// dependent launch; off with DMR_PDL=0).  Such a kernel calls pdl_wait() before it touches anything an earlier kernel of
+// the stream wrote, and pdl_launch_dependents() once its own successor may start.
+bool tc_pdl_enabled();
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = tc_pdl_enabled() ? 1u : 0u;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif  // __CUDACC__

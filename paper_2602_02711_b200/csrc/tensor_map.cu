@@ -5,6 +5,8 @@
 #include <mutex>
 #include <unordered_map>
 
+#include <cstdlib>
+
 #include "sm100.cuh"
 
 namespace dmr {
@@ -93,6 +95,15 @@ bool ensure_dynamic_smem(const void *kernel, size_t bytes) {
     }
     done[key] = bytes;
     return true;
+}
+
+bool tc_pdl_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("DMR_PDL");
+        v = (e && e[0] == '0') ? 0 : 1;
+    }
+    return v != 0;
 }
 
 }  // namespace dmr
