@@ -57,23 +57,22 @@ struct PrefillCfg {
 // Largest magnitude pattern among a feature's G bf16 scales (sign bit cleared): eight scales per 16-byte load when the
 // row of the table allows it, so that a work item's set-up is a handful of independent loads, not a chain of G.
 __device__ __forceinline__ uint32_t scale_row_max(const uint16_t *sp, int G) {
-    uint32_t smax = 0;
-    if ((G & 7) == 0 && (reinterpret_cast<uintptr_t>(sp) & 15) == 0) {
-        uint32_t m0 = 0, m1 = 0;
-        for (int gi = 0; gi < G; gi += 8) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(sp + gi));
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t m0 = 0, m1 = 0;
+    int gi = 0;
+    // scalar loads up to the first 16-byte boundary, 16-byte loads over the aligned middle, scalar loads for the rest
+    const int head = (int)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(sp) & 15u)) & 15u) >> 1);
+    for (; gi < G && gi < head; ++gi) m0 = max(m0, (uint32_t)__ldg(sp + gi) & 0x7FFFu);
+    for (; gi + 8 <= G; gi += 8) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(sp + gi));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                m0 = max(m0, w[i] & 0x7FFFu);
-                m1 = max(m1, (w[i] >> 16) & 0x7FFFu);
-            }
+        for (int i = 0; i < 4; ++i) {
+            m0 = max(m0, w[i] & 0x7FFFu);
+            m1 = max(m1, (w[i] >> 16) & 0x7FFFu);
         }
-        smax = max(m0, m1);
-    } else {
-        for (int gi = 0; gi < G; ++gi) smax = max(smax, (uint32_t)__ldg(sp + gi) & 0x7FFFu);
     }
-    return smax;
+    for (; gi < G; ++gi) m1 = max(m1, (uint32_t)__ldg(sp + gi) & 0x7FFFu);
+    return max(m0, m1);
 }
 
 struct PrefillArgs {
