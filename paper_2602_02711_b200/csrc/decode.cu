@@ -1,5 +1,5 @@
-// Decode-time 4-bit linear layer (up to 16 rows per launch): the weight matrix is read exactly once at memory
-// speed.  Decoding re-streams the model weights for every generated token and is limited by memory
+// Decode-time 4-bit (and 3-bit) linear layer (up to 16 rows per launch): the weight matrix is read exactly once.
+// Decoding re-streams the model weights for every generated token and is limited by memory
 // bandwidth, which is where weight-only quantization pays (App. "Evaluation protocol", discussion of output
 // length; App. "Latency coefficients").
 //
@@ -8,23 +8,28 @@
 // there is no scratch memory, no counter and no wait on another CTA in this kernel.  Inside the CTA all warps
 // work on the same tile and split its k range in boxes of 256 input features (box b goes to warp b % WARPS).
 // The partial sums of every output are added in warp order through shared memory - a fixed order that depends
-// on the instance and the layer's shape only, so a row's result never depends on the batch around it.
+// on the instance and the layer's shape only, so a row's result never depends on the batch around it.  The hand-over
+// is by mbarrier: a warp announces its sums of a tile and adds up the tile before, so the loop has no CTA-wide barrier.
 //
 // Data movement.  Every warp has a ring of its own in shared memory that one of its lanes keeps full with TMA
 // boxes of [16 R rows x 128 bytes] of packed codes (two or four chunks; rows past N read as zero; 128-byte
-// swizzle); nobody else reads it, so the only synchronisation is the warp's own mbarrier per stage.  The boxes
+// swizzle; 3-bit codes: rows of 96 bytes, not swizzled); nobody else reads it, so the only synchronisation is
+// the warp's own mbarrier per stage.  The boxes
 // are as large as the tile allows because every box costs the SM's copy engine a fixed time of its own
 // (measured: about 70 cycles, whatever its size).  A tile's scales and zero points are two contiguous blocks
-// of the tables; one thread copies them to shared memory two tiles ahead (bulk copies) when the layer's shape
+// of the tables; one thread copies them to shared memory three tiles ahead (bulk copies) when the layer's shape
 // allows it, otherwise they are read from global memory where they are needed.  Activations come through the
-// L1 with ordinary loads issued one chunk ahead.
+// L1 with ordinary loads issued a chunk's worth of arithmetic ahead, piece by piece as their registers fall free.
 //
 // Inner loop.  Lane (g, t) (g = lane / 4, t = lane % 4) takes WPL consecutive code words of two rows of each
 // 16-row block and the 8 WPL activations they meet for batch rows g (and g + 8 in the 16-row instance).
 // ((w >> 4p) & 0x000F000F) | 0x43004300 is the bf16 pair {128 + q_p, 128 + q_{p+4}} - exact - and goes to the
 // tensor cores as it is (mma.m16n8k16, the weights as the 16-row operand), a byte permute pairs the
-// activations the same way, and one more MMA with an all-ones operand gives the sum of the chunk's activations
-// per batch row.  A chunk never crosses a quantization group, so per chunk
+// activations the same way, and MMAs with an all-ones operand give the sum of the chunk's activations per batch
+// row (the common layer shapes form these sums in the CTA's first tile only and keep them in shared memory: they do
+// not depend on the tile).  3-bit codes: 32 codes in three words, five per half-word - (w >> 3i) & 0x00070007 is the
+// pair of codes i and i + 5 of a word, the pair at bits 3..5 is taken unshifted as 128 + 8 q and brought to 128 + q by
+// one bf16 fma.  A chunk never crosses a quantization group, so per chunk
 //     sum_k x_k s (q_k - z) = s (sum_k x_k (128 + q_k) - (128 + z) sum_k x_k)
 // is formed in fp32 from the two accumulators: no weight is rounded, the zero point costs nothing per weight,
 // and the error against exact arithmetic is fp32 summation of terms about thirty times the result (a few
@@ -34,7 +39,8 @@
 // more than half of an SM's shared memory, so that an SM never holds two CTAs of these kernels: the
 // successor's CTA moves in when this kernel's CTA on that SM has finished, fills its rings and only then waits
 // for its predecessor.  (Bulk prefetches of the CTA's whole share into the L2 were tried on top of the rings and
-// cost more issue slots than they saved: 159 against 147 us per sweep of twelve layers.)  (With two CTAs per SM the successor's CTAs land wherever a slot happens to be free - two on
+// cost more issue slots than they saved: 159 against 147 us per sweep of twelve layers.)  (With two CTAs per SM
+// the successor's CTAs land wherever a slot happens to be free - two on
 // some SMs, none on others - and the kernel runs at the pace of the doubly loaded SMs; measured with in-kernel
 // time stamps.)  Weights, scales and zero points are read before the wait: they must not be produced by a
 // kernel that releases its dependents early (the library's own kernels that write weights never do).
