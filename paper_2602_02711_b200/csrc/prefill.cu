@@ -417,24 +417,30 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 } else {
                     const float zf = __uint_as_float(0x4B000000u | zb);  // 2^23 + zero
                     const float sf = __uint_as_float(sb << 16) * fdown;
+                    // A row of codes is 64 bytes = four 16-byte pieces.  Lane r starts at piece (r / 2) % 4, so that the eight
+                    // lanes of a load phase read eight different bank groups (all starting at piece 0 would meet in two).
+                    // Piece q holds codes 16 q .. 16 q + 15 = chunks 2 q and 2 q + 1 of the fp16 row.
 #pragma unroll
-                    for (int cc = 0; cc < CH; ++cc) {  // chunk c = codes 8c .. 8c+7 = packed words 2c, 2c+1
-                        const int c = c_lo + cc;
-                        uint32_t w0, w1;
-                        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(w0), "=r"(w1) : "r"(src + 8 * c));
-                        uint32_t o[4];
+                    for (int j = 0; j < CH / 2; ++j) {
+                        const uint32_t q = ((uint32_t)j + (uint32_t)(r >> 1)) & 3u;
+                        uint32_t wq[4];
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(wq[0]), "=r"(wq[1]), "=r"(wq[2]), "=r"(wq[3]) : "r"(src + 16u * q));
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const uint32_t u = h ? w1 : w0;
-                            float f[4];
+                        for (int e = 0; e < 2; ++e) {
+                            uint32_t o[4];
 #pragma unroll
-                            for (int b = 0; b < 4; ++b)  // (q - zero) exactly, times the scale exactly (8 x 8 bits)
-                                f[b] = __fmul_rn(__fsub_rn(__uint_as_float(prmt(u, 0x4B000000u, 0x7650u + (uint32_t)b)), zf), sf);
-                            o[2 * h] = pack_f16x2_rn(f[0], f[1]);  // the one rounding
-                            o[2 * h + 1] = pack_f16x2_rn(f[2], f[3]);
+                            for (int h = 0; h < 2; ++h) {
+                                const uint32_t u = wq[2 * e + h];
+                                float f[4];
+#pragma unroll
+                                for (int b = 0; b < 4; ++b)  // (q - zero) exactly, times the scale exactly (8 x 8 bits)
+                                    f[b] = __fmul_rn(__fsub_rn(__uint_as_float(prmt(u, 0x4B000000u, 0x7650u + (uint32_t)b)), zf), sf);
+                                o[2 * h] = pack_f16x2_rn(f[0], f[1]);  // the one rounding
+                                o[2 * h + 1] = pack_f16x2_rn(f[2], f[3]);
+                            }
+                            const uint32_t addr = dst + (((2u * q + (uint32_t)e) ^ swz) << 4);
+                            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
                         }
-                        const uint32_t addr = dst + ((((uint32_t)c) ^ swz) << 4);
-                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
                     }
                 }
                 fence_proxy_async_smem();  // the tile must be visible to the tensor core's reads
