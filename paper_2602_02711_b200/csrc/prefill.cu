@@ -4,7 +4,7 @@
 // belongs on the tensor cores.
 //
 // Orientation: the weights are the 128-row operand (D[n][m] = sum_k W^[n][k] X[m][k]), one
-// tensor-memory lane per output feature, BN (128 or 256) activation rows as the N operand.
+// tensor-memory lane per output feature, BN (64, 128 or 256) activation rows as the N operand.
 //
 // Per 64-wide k block and stage of the ring:
 //   warp 0      TMA: the packed code tile [128 features x 32 or 64 bytes] and the activation tile
@@ -27,6 +27,8 @@
 // epilogue multiplies the two powers of two back in (exact).
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "sm100.cuh"
 
 namespace dmr {
@@ -48,8 +50,8 @@ struct PrefillCfg {
     static constexpr int S = S_RAW > 8 ? 8 : S_RAW;
     static constexpr int TMEM_COLS = 2 * BN;                 // two accumulators
     // unpack warps: UW / 4 groups of four, group i takes every (UW / 4)-th stage of the ring.  Three groups for the
-    // 128-row tile (small batches: a stage's MMAs are short and the unpack chain's latency is what is left), two for 256.
-    static constexpr int UW = BN == 128 ? 12 : 8;
+    // 64- and 128-row tiles (small batches: a stage's MMAs are short and the unpack chain's latency is what is left), two for 256.
+    static constexpr int UW = BN == 256 ? 8 : 12;
     static constexpr int THREADS = 32 * (2 + UW + 4);
     static constexpr size_t SMEM = (size_t)S * STAGE + 1024 /*alignment*/ + 512 /*barriers*/;
 };
@@ -482,17 +484,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(buf));
                 }
-                if (n < a.N) {
+                // Row scales and (routed calls) output rows of this block of 32 batch slots: one coalesced load each, handed
+                // round by shuffles.  (A load per element inside the guarded loop below is a chain of 32 exposed round trips.)
+                const int m_lane = m0 + c0 + lane;
+                const float xs_lane = m_lane < rows ? __ldg(a.xscale + m_lane) : 0.f;
+                const int row_lane = (!SPLITK && a.idx && m_lane < rows) ? a.idx[m_lane] : m_lane;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const int m = m0 + c0 + c;
-                        if (m < rows) {
-                            const float v = (__uint_as_float(u[c]) * __ldg(a.xscale + m)) * fscale;
-                            if constexpr (SPLITK) {  // this split's share, by batch slot; the reduction scatters the rows
-                                a.partial[((size_t)split * a.M + m) * a.N + n] = v;
-                                continue;
-                            }
-                            const int row = a.idx ? a.idx[m] : m;
+                for (int c = 0; c < 32; ++c) {
+                    const float xs = __shfl_sync(0xffffffffu, xs_lane, c);
+                    const int row = __shfl_sync(0xffffffffu, row_lane, c);
+                    const int m = m0 + c0 + c;
+                    if (n < a.N && m < rows) {
+                        const float v = (__uint_as_float(u[c]) * xs) * fscale;
+                        if constexpr (SPLITK) {  // this split's share, by batch slot; the reduction scatters the rows
+                            a.partial[((size_t)split * a.M + m) * a.N + n] = v;
+                        } else {
                             if (OUT_F32) reinterpret_cast<float *>(a.Y)[(size_t)row * a.N + n] = v;
                             else reinterpret_cast<__nv_bfloat16 *>(a.Y)[(size_t)row * a.N + n] = __float2bfloat16_rn(v);
                         }
@@ -545,7 +551,8 @@ int prefill_sm_count() {
 // Activation rows per tile: 256 halves the unpack work and shared-memory traffic per flop, 128 fills
 // the last wave better when there are few tiles.  Depends on (M, N) only.
 int prefill_bn(int M, int N, int sms) {
-    if (M <= 128) return 128;  // one tile of rows: the smaller activation tile leaves room for more stages
+    if (M <= 64) return 64;    // one tile of rows: the smaller the activation tile, the more stages are in flight
+    if (M <= 128) return 128;
     const int n_tiles = (N + PM - 1) / PM;
     auto score = [&](int bn, double rate) {
         const long long t = (long long)n_tiles * ((M + bn - 1) / bn);
@@ -655,9 +662,15 @@ dmr_status_t launch_prefill(const uint16_t *X, int M, RowSel sel, const void *qw
     const long long tiles = (long long)a.n_tiles * a.m_tiles * splits;
     const int grid = (int)(tiles < sms ? tiles : sms);
     dmr_status_t r;
-    if (bits == 3) r = bn == 256 ? launch_prefill_t<3, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<3, 128>(map_w, map_x, a, grid, out, st);
-    else if (bits == 4) r = bn == 256 ? launch_prefill_t<4, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<4, 128>(map_w, map_x, a, grid, out, st);
-    else r = bn == 256 ? launch_prefill_t<8, 256>(map_w, map_x, a, grid, out, st) : launch_prefill_t<8, 128>(map_w, map_x, a, grid, out, st);
+    auto by_rows = [&](auto bits_tag) -> dmr_status_t {
+        constexpr int B = decltype(bits_tag)::value;
+        if (bn == 256) return launch_prefill_t<B, 256>(map_w, map_x, a, grid, out, st);
+        if (bn == 128) return launch_prefill_t<B, 128>(map_w, map_x, a, grid, out, st);
+        return launch_prefill_t<B, 64>(map_w, map_x, a, grid, out, st);
+    };
+    if (bits == 3) r = by_rows(std::integral_constant<int, 3>{});
+    else if (bits == 4) r = by_rows(std::integral_constant<int, 4>{});
+    else r = by_rows(std::integral_constant<int, 8>{});
     if (r != DMR_OK || splits == 1) return r;
     return launch_splitk_reduce(partial, splits, M, N, sel, Y, out, st);
 }
