@@ -134,6 +134,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         // ================= MMA issuer =================
         if (lane == 0) {
             constexpr uint32_t IDESC = umma_idesc_bf16(BM, BN);
+            // operand descriptors of stage 0; a stage and a k step only move the address field (16-byte units)
+            const uint64_t desc_a0 = umma_desc_sw128(a_tile(0)), desc_b0 = umma_desc_sw128(b_tile(0));
             int buf = 0, groups_done = 0;
             bool group_start = true;
             for (int i = 0; i < nkb; ++i) {
@@ -147,12 +149,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 }
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                const uint64_t stage_off = (uint64_t)(((uint32_t)s * (uint32_t)Cfg::STAGE_BYTES) >> 4);
 #pragma unroll
-                for (int j = 0; j < BK / 16; ++j) {
-                    const uint64_t adesc = umma_desc_sw128(a_tile(s) + j * 32);
-                    const uint64_t bdesc = umma_desc_sw128(b_tile(s) + j * 32);
-                    umma_bf16_ss(d_tmem, adesc, bdesc, IDESC, (group_start && j == 0) ? 0u : 1u);
-                }
+                for (int j = 0; j < BK / 16; ++j)  // 16 k values = 32 bytes of a row = two 16-byte units
+                    umma_bf16_ss(d_tmem, desc_a0 + stage_off + (uint64_t)(2 * j), desc_b0 + stage_off + (uint64_t)(2 * j), IDESC,
+                                 (group_start && j == 0) ? 0u : 1u);
                 umma_commit(empty_bar(s));
                 group_start = false;
                 const int kb = kb_begin + i;

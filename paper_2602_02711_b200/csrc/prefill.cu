@@ -258,6 +258,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // ================= MMA issuer =================
         if (lane == 0) {
             constexpr uint32_t IDESC = umma_idesc_f16(PM, BN);
+            // Operand descriptors: built once for stage 0; a stage and a k step only move the 14-bit address field (16-byte
+            // units), so each MMA costs this one thread an add, not a descriptor's worth of dependent shifts and ORs.
+            const uint64_t desc_a0 = umma_desc_sw128(a_tile(0)), desc_b0 = umma_desc_sw128(b_tile(0));
             uint32_t it = 0, tile_it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
@@ -274,9 +277,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         break;
                     }
                     tcgen05_fence_after();
+                    const uint64_t stage_off = (uint64_t)(((uint32_t)s * (uint32_t)Cfg::STAGE) >> 4);
+                    const uint64_t desc_a = desc_a0 + stage_off, desc_b = desc_b0 + stage_off;
 #pragma unroll
-                    for (int j = 0; j < PK / 16; ++j)
-                        umma_bf16_ss(d_tmem, umma_desc_sw128(a_tile(s) + j * 32), umma_desc_sw128(b_tile(s) + j * 32), IDESC,
+                    for (int j = 0; j < PK / 16; ++j)  // 16 k values = 32 bytes of a row = two 16-byte units
+                        umma_bf16_ss(d_tmem, desc_a + (uint64_t)(2 * j), desc_b + (uint64_t)(2 * j), IDESC,
                                      (kb == kb_lo && j == 0) ? 0u : 1u);
                     umma_commit(empty_bar(s));
                 }
