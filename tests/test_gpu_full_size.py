@@ -92,6 +92,20 @@ def test_prefill_many_tiles_per_cta_with_ragged_features():
     assert dmr.dmr_describe_dispatch(OP_LOWBIT, 1024, 12288, 4096, QFormat(4, 128))["tiles"] >= 2 * 148
 
 
+@pytest.mark.parametrize("bits", [4, 3])
+def test_prefill_64_row_tile_several_tiles_per_cta(bits):
+    # up to 64 rows run the 64-row instance; 40000 features = 313 feature tiles (the last one ragged) on 148 CTAs,
+    # no split along k: every CTA runs two or three tiles back to back through both accumulators
+    M, N, K = 50, 40000, 1024
+    plan = dmr.dmr_describe_dispatch(OP_LOWBIT, M, N, K, QFormat(bits, 128))
+    assert plan["kernel"] == "prefill" and plan["bn"] == 64 and plan["splits"] == 1 and plan["tiles"] > 2 * plan["ctas"]
+    W, q, ref = quantized_layer(N, K, bits, 128, seed=43)
+    X = inputs.activations(M, K, seed=43, index=M)
+    Y32 = dmr.dmr_lowbit_linear(to_dev_bf16(X), q, OUT_F32)
+    ms, ns, want, scale = sampled_reference(X, M, N, 43, qweight=ref[0], scales=ref[1], zeros=ref[2], bits=bits, group=128)
+    check(Y32, ms, ns, want, scale, TOL_PREFILL)
+
+
 # ---------------- streaming kernel with feature groups split across CTAs (no clusters) ----------------
 
 @pytest.mark.parametrize("M,out", [(1, OUT_F32), (16, OUT_BF16), (27, OUT_F32)])
