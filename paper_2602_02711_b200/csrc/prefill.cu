@@ -9,13 +9,14 @@
 // Per 64-wide k block and stage of the ring:
 //   warp 0      TMA: the packed code tile [128 features x 32 or 64 bytes] and the activation tile
 //               [BN rows x 128 bytes, 128-byte swizzle] land in shared memory (one mbarrier);
-//   warps 2..9 (2..13 for the 128-row tile)  one thread per feature row turns its codes into the fp16 weights s' * (q - zero)
+//   warps 2..9 (2..13 for the 64- and 128-row tiles)  one thread per feature row turns its codes into the fp16 weights s' * (q - zero)
 //               (exact integer q - zero, then ONE rounding of the product to 11 significant bits)
 //               and stores them as the swizzled K-major A tile;
 //   warp 1      one lane issues four tcgen05.mma (128 x BN x 16) that accumulate into one of two
 //               fp32 accumulators in tensor memory, and commits the stage back to the producer;
 //   the last four warps drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
-//               next tile's MMAs run into the other accumulator.
+//               next tile's MMAs run into the other accumulator (a block of 32 rows at a time: the rows' scales and
+//               output rows come from one coalesced load each, never from loads inside the store loop).
 // CTAs are persistent: CTA b takes tiles b, b + grid, ...  Every wait is bounded.
 //
 // Operand precision.  The MMA runs in fp16 x fp16 -> fp32 (kind::f16) instead of bf16: a bf16 A
