@@ -554,18 +554,20 @@ int prefill_sm_count() {
     return cached;
 }
 
-// Activation rows per tile: 256 halves the unpack work and shared-memory traffic per flop, 128 fills
-// the last wave better when there are few tiles.  Depends on (M, N) only.
+// Activation rows per tile.  A k block costs a CTA about the same time whatever the tile's width (hand-overs between the
+// roles, not MMA time, set the pace), so the wide tile does about twice the work per unit of time; the narrow one is
+// for batches it covers alone and for shapes whose last wave it fills much better.  Depends on (M, N) only.
 int prefill_bn(int M, int N, int sms) {
     if (M <= 64) return 64;    // one tile of rows: the smaller the activation tile, the more stages are in flight
     if (M <= 128) return 128;
     const int n_tiles = (N + PM - 1) / PM;
     auto score = [&](int bn, double rate) {
         const long long t = (long long)n_tiles * ((M + bn - 1) / bn);
+        if (t < sms) return rate;  // fewer tiles than SMs: split along k fills the SMs (prefill_splits)
         const long long waves = (t + sms - 1) / sms;
         return rate * (double)t / (double)(waves * sms);
     };
-    return score(256, 1.0) >= score(128, 0.8) ? 256 : 128;
+    return score(256, 1.0) >= score(128, 0.7) ? 256 : 128;  // (measured: the narrow tile wins between 0.67 and 0.75)
 }
 
 }  // namespace
@@ -578,15 +580,18 @@ bool prefill_supported(int M, int N, int K, int bits, int g) {
     return M > 32 && (N + PM - 1) / PM >= 16;
 }
 
-// Split-K factor: only for a single row tile (M <= 128) on layers whose feature tiles leave SMs idle.  As many splits
-// as give every SM at most one work item, each with at least sixteen k blocks.  Depends on (M, N, K) only.
+// Split-K factor: for shapes whose tiles leave SMs idle.  As many splits as give every SM at most one work item, each
+// with at least sixteen k blocks; with more than one row tile the fp32 partial sums are large, and a split is taken only
+// if it shortens a work item by at least 48 k blocks.  Depends on (M, N, K) only.
 static int prefill_splits(int M, int N, int K, int sms, int *kb_per_split) {
-    const int nkb = K / PK, tiles = (N + PM - 1) / PM;
+    const int bn = prefill_bn(M, N, sms);
+    const int nkb = K / PK, tiles = ((N + PM - 1) / PM) * ((M + bn - 1) / bn);
     int splits = 1;
-    if (M <= 128 && tiles < sms) {
+    if (tiles < sms) {
         splits = sms / tiles;
         if (splits > nkb / 16) splits = nkb / 16;  // a work item pays for its set-up (the feature's scale range) once
         if (splits < 1) splits = 1;
+        if (M > 128 && nkb - (nkb + splits - 1) / splits < 48) splits = 1;
     }
     *kb_per_split = (nkb + splits - 1) / splits;
     return (nkb + *kb_per_split - 1) / *kb_per_split;  // no empty split

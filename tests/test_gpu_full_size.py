@@ -92,6 +92,23 @@ def test_prefill_many_tiles_per_cta_with_ragged_features():
     assert dmr.dmr_describe_dispatch(OP_LOWBIT, 1024, 12288, 4096, QFormat(4, 128))["tiles"] >= 2 * 148
 
 
+def test_prefill_split_k_over_two_row_tiles():
+    # 300 rows = two 256-row tiles (the second ragged) x 32 feature tiles leave SMs idle: every tile's k range is split in
+    # two work items, fp32 partial sums added in split order by the second kernel
+    name, M = "down", 300
+    N, K = inputs.LAYER_7B[name]
+    plan = dmr.dmr_describe_dispatch(OP_LOWBIT, M, N, K, QFormat(4, 128))
+    assert plan["kernel"] == "prefill" and plan["bn"] == 256 and plan["splits"] == 2 and plan["tiles"] == 64
+    W, q, ref = quantized_layer(N, K, 4, 128, seed=40)
+    X = inputs.activations(M, K, seed=44, index=M)
+    Xd = to_dev_bf16(X)
+    Y32 = dmr.dmr_lowbit_linear(Xd, q, OUT_F32)
+    ms, ns, want, scale = sampled_reference(X, M, N, 44, qweight=ref[0], scales=ref[1], zeros=ref[2], bits=4, group=128)
+    check(Y32, ms, ns, want, scale, TOL_PREFILL)
+    assert torch.equal(dmr.dmr_lowbit_linear(Xd, q, OUT_BF16), Y32.to(torch.bfloat16))
+    assert torch.equal(dmr.dmr_lowbit_linear(Xd, q, OUT_F32), Y32)  # the sum order is fixed: repeatable bit for bit
+
+
 @pytest.mark.parametrize("bits", [4, 3])
 def test_prefill_64_row_tile_several_tiles_per_cta(bits):
     # up to 64 rows run the 64-row instance; 40000 features = 313 feature tiles (the last one ragged) on 148 CTAs,
