@@ -132,7 +132,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        // the whole warp runs the loop (the same stage numbers and descriptors in all lanes), one lane issues
+        {
             constexpr uint32_t IDESC = umma_idesc_bf16(BM, BN);
             // operand descriptors of stage 0; a stage and a k step only move the address field (16-byte units)
             const uint64_t desc_a0 = umma_desc_sw128(a_tile(0)), desc_b0 = umma_desc_sw128(b_tile(0));
@@ -150,16 +151,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ C
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 const uint64_t stage_off = (uint64_t)(((uint32_t)s * (uint32_t)Cfg::STAGE_BYTES) >> 4);
+                if (lane == 0) {
 #pragma unroll
-                for (int j = 0; j < BK / 16; ++j)  // 16 k values = 32 bytes of a row = two 16-byte units
-                    umma_bf16_ss(d_tmem, desc_a0 + stage_off + (uint64_t)(2 * j), desc_b0 + stage_off + (uint64_t)(2 * j), IDESC,
-                                 (group_start && j == 0) ? 0u : 1u);
-                umma_commit(empty_bar(s));
+                    for (int j = 0; j < BK / 16; ++j)  // 16 k values = 32 bytes of a row = two 16-byte units
+                        umma_bf16_ss(d_tmem, desc_a0 + stage_off + (uint64_t)(2 * j), desc_b0 + stage_off + (uint64_t)(2 * j), IDESC,
+                                     (group_start && j == 0) ? 0u : 1u);
+                    umma_commit(empty_bar(s));
+                }
+                __syncwarp();
                 group_start = false;
                 const int kb = kb_begin + i;
                 const bool group_end = LOWBIT ? (((kb + 1) % kb_per_group) == 0 || i == nkb - 1) : (i == nkb - 1);
                 if (group_end) {
-                    umma_commit(tfull_bar(buf));
+                    if (lane == 0) umma_commit(tfull_bar(buf));
+                    __syncwarp();
                     if (LOWBIT) buf ^= 1;
                     ++groups_done;
                     group_start = true;

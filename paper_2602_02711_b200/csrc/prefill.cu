@@ -257,11 +257,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        // The whole warp runs the loop: stage numbers, descriptors and accumulator addresses are then the same in all
+        // lanes (the compiler can keep them in uniform registers, which the MMA instruction reads), and one lane issues.
+        {
             constexpr uint32_t IDESC = umma_idesc_f16(PM, BN);
             // Operand descriptors: built once for stage 0; a stage and a k step only move the 14-bit address field (16-byte
-            // units), so each MMA costs this one thread an add, not a descriptor's worth of dependent shifts and ORs.
+            // units), so each MMA costs an add, not a descriptor's worth of dependent shifts and ORs.
             const uint64_t desc_a0 = umma_desc_sw128(a_tile(0)), desc_b0 = umma_desc_sw128(b_tile(0));
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
             uint32_t it = 0, tile_it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
@@ -269,7 +272,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 // the epilogue must have drained this accumulator (used two tiles ago)
                 if (tile_it >= 2 && !mbar_wait(tempty_bar(buf), ((tile_it >> 1) - 1) & 1, a.status)) break;
                 tcgen05_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                const uint32_t d_tmem = tmem_u + (uint32_t)(buf * BN);
                 const int kb_lo = SPLITK ? (tile % n_splits) * a.kb_per_split : 0, kb_hi = SPLITK ? min(nkb, kb_lo + a.kb_per_split) : nkb;
                 for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
                     const int s = it % S;
@@ -280,13 +283,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     tcgen05_fence_after();
                     const uint64_t stage_off = (uint64_t)(((uint32_t)s * (uint32_t)Cfg::STAGE) >> 4);
                     const uint64_t desc_a = desc_a0 + stage_off, desc_b = desc_b0 + stage_off;
+                    if (lane == 0) {
 #pragma unroll
-                    for (int j = 0; j < PK / 16; ++j)  // 16 k values = 32 bytes of a row = two 16-byte units
-                        umma_bf16_ss(d_tmem, desc_a + (uint64_t)(2 * j), desc_b + (uint64_t)(2 * j), IDESC,
-                                     (kb == kb_lo && j == 0) ? 0u : 1u);
-                    umma_commit(empty_bar(s));
+                        for (int j = 0; j < PK / 16; ++j)  // 16 k values = 32 bytes of a row = two 16-byte units
+                            umma_bf16_ss(d_tmem, desc_a + (uint64_t)(2 * j), desc_b + (uint64_t)(2 * j), IDESC,
+                                         (kb == kb_lo && j == 0) ? 0u : 1u);
+                        umma_commit(empty_bar(s));
+                    }
+                    __syncwarp();
                 }
-                if (ok) umma_commit(tfull_bar(buf));
+                if (ok && lane == 0) umma_commit(tfull_bar(buf));
+                __syncwarp();
             }
         }
     } else if (warp < 2 + Cfg::UW) {
