@@ -324,6 +324,35 @@ splitk_reduce_kernel(const float *__restrict__ partial, int splits, int M, int N
     pdl_wait();  // the partial sums come from the kernel before this one
     pdl_launch_dependents();
     const int rows = count ? min(*count, M) : M;
+    if ((N & 3) == 0 && (size_t)rows * (size_t)N < 0x7FFFFFFFull) {
+        // four consecutive features per thread: 16-byte loads of every split's sums, one 8- or 16-byte store
+        const unsigned nq = (unsigned)N >> 2, total = (unsigned)rows * nq;
+        const size_t zstride = (size_t)M * (size_t)N / 4;
+        for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+            const unsigned m = i / nq, q = i - m * nq;
+            const int row = idx ? idx[m] : (int)m;
+            const float4 *p = reinterpret_cast<const float4 *>(partial) + (size_t)m * nq + q;
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int z = 0; z < splits; ++z) {  // in split order, as the one-element path below
+                const float4 v = p[(size_t)z * zstride];
+                s.x += v.x;
+                s.y += v.y;
+                s.z += v.z;
+                s.w += v.w;
+            }
+            const size_t o = (size_t)row * N + 4u * q;
+            if (OUT_F32) {
+                *reinterpret_cast<float4 *>(reinterpret_cast<float *>(Y) + o) = s;
+            } else {
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(s.x, s.y), hi = __floats2bfloat162_rn(s.z, s.w);
+                uint2 w;
+                w.x = *reinterpret_cast<const uint32_t *>(&lo);
+                w.y = *reinterpret_cast<const uint32_t *>(&hi);
+                *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(Y) + o) = w;
+            }
+        }
+        return;
+    }
     const size_t total = (size_t)rows * N;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const int m = (int)(i / N), n = (int)(i % N);
@@ -458,22 +487,13 @@ dmr_status_t launch_gemm(const uint16_t *X, int M, RowSel sel, const void *weigh
     else if (bits == 4) r = launch_gemm_bn<4>(p.bn, map_w, map_x, a, p.splits, out, st);
     else r = launch_gemm_bn<8>(p.bn, map_w, map_x, a, p.splits, out, st);
     if (r != DMR_OK) return r;
-    if (p.splits > 1) {
-        const size_t total = (size_t)M * N;
-        int blocks = (int)((total + 255) / 256);
-        if (blocks > 148 * 8) blocks = 148 * 8;
-        if (out == DMR_OUT_F32)
-            (void)launch_pdl(splitk_reduce_kernel<true>, dim3((unsigned)blocks), dim3(256), 0, st, partial, p.splits, M, N, sel.idx, sel.count, Y);
-        else
-            (void)launch_pdl(splitk_reduce_kernel<false>, dim3((unsigned)blocks), dim3(256), 0, st, partial, p.splits, M, N, sel.idx, sel.count, Y);
-        r = check_launch();
-    }
+    if (p.splits > 1) r = launch_splitk_reduce(partial, p.splits, M, N, sel, Y, out, st);
     return r;
 }
 
 dmr_status_t launch_splitk_reduce(const float *partial, int splits, int M, int N, RowSel sel, void *Y, dmr_out_t out,
                                   cudaStream_t st) {
-    const size_t total = (size_t)M * N;
+    const size_t total = (size_t)M * N / ((N & 3) == 0 ? 4 : 1);
     int blocks = (int)((total + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
     if (out == DMR_OUT_F32)
