@@ -144,6 +144,7 @@ def test_config1_lowbit_linear(M):
     (40, 300, 512, 4, 128),    # M above the decode limit: tensor-core GEMM, ragged N and M
     (33, 136, 384, 8, 0),
     (64, 256, 4096, 4, 128),   # few tiles, long K: split-K with ordered reduction
+    (64, 250, 4096, 4, 128),   # ... and N not a multiple of 4: the sums of the splits go one feature per thread
     (130, 264, 1024, 4, 64),   # two column blocks, g = 64
     (100, 200, 2048, 8, 0),    # INT8 per-channel: one group spans all of K
     (300, 520, 640, 4, 128),
