@@ -497,18 +497,31 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(buf));
                 }
-                // Row scales and (routed calls) output rows of this block of 32 batch slots: one coalesced load each, handed
-                // round by shuffles.  (A load per element inside the guarded loop below is a chain of 32 exposed round trips.)
+                // Row scales of this block of 32 batch slots: eight 16-byte loads from one address for the whole warp (the table
+                // is padded to a multiple of 64 entries).  A load per element inside the guarded loop below would be a chain of
+                // 32 exposed round trips, and every shuffle or load is one more instruction through the memory pipe, which the
+                // operand tiles keep busy.  Output rows of a routed call: one coalesced load, handed round by shuffles.
+                float xs[32];
+                {
+                    const float4 *xp = reinterpret_cast<const float4 *>(a.xscale + m0 + c0);
+#pragma unroll
+                    for (int q4 = 0; q4 < 8; ++q4) {
+                        const float4 t = __ldg(xp + q4);
+                        xs[4 * q4] = t.x;
+                        xs[4 * q4 + 1] = t.y;
+                        xs[4 * q4 + 2] = t.z;
+                        xs[4 * q4 + 3] = t.w;
+                    }
+                }
+                const bool listed = !SPLITK && a.idx != nullptr;
                 const int m_lane = m0 + c0 + lane;
-                const float xs_lane = m_lane < rows ? __ldg(a.xscale + m_lane) : 0.f;
-                const int row_lane = (!SPLITK && a.idx && m_lane < rows) ? a.idx[m_lane] : m_lane;
+                const int row_lane = (listed && m_lane < rows) ? a.idx[m_lane] : m_lane;
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
-                    const float xs = __shfl_sync(0xffffffffu, xs_lane, c);
-                    const int row = __shfl_sync(0xffffffffu, row_lane, c);
                     const int m = m0 + c0 + c;
+                    const int row = listed ? __shfl_sync(0xffffffffu, row_lane, c) : m;
                     if (n < a.N && m < rows) {
-                        const float v = (__uint_as_float(u[c]) * xs) * fscale;
+                        const float v = (__uint_as_float(u[c]) * xs[c]) * fscale;
                         if constexpr (SPLITK) {  // this split's share, by batch slot; the reduction scatters the rows
                             a.partial[((size_t)split * a.M + m) * a.N + n] = v;
                         } else {
