@@ -14,7 +14,8 @@
 //               and stores them as the swizzled K-major A tile;
 //   warp 1      one lane issues four tcgen05.mma (128 x BN x 16) that accumulate into one of two
 //               fp32 accumulators in tensor memory, and commits the stage back to the producer;
-//   the last four warps drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
+//   the last four warps (eight for the 256-row tile, two per lane quadrant with half of the columns each)
+//               drain the finished accumulator of the previous tile (tcgen05.ld) into Y while the
 //               next tile's MMAs run into the other accumulator (a block of 32 rows at a time: the rows' scales and
 //               output rows come from one coalesced load each, never from loads inside the store loop).
 // CTAs are persistent: CTA b takes tiles b, b + grid, ...  Every wait is bounded.
@@ -53,7 +54,10 @@ struct PrefillCfg {
     // unpack warps: UW / 4 groups of four, group i takes every (UW / 4)-th stage of the ring.  Three groups for the
     // 64- and 128-row tiles (small batches: a stage's MMAs are short and the unpack chain's latency is what is left), two for 256.
     static constexpr int UW = BN == 256 ? 8 : 12;
-    static constexpr int THREADS = 32 * (2 + UW + 4);
+    // epilogue warps: four (one per tensor-memory lane quadrant), eight for the 256-row tile (two per quadrant, each draining
+    // half of the accumulator's columns: what is left after a CTA's last MMA is its last tile's epilogue)
+    static constexpr int EW = BN == 256 ? 8 : 4;
+    static constexpr int THREADS = 32 * (2 + UW + EW);
     static constexpr size_t SMEM = (size_t)S * STAGE + 1024 /*alignment*/ + 512 /*barriers*/;
 };
 
@@ -206,7 +210,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull_bar(b), 1);
-            mbar_init(tempty_bar(b), 4);  // one arrival per epilogue warp
+            mbar_init(tempty_bar(b), Cfg::EW);  // one arrival per epilogue warp
         }
         fence_barrier_init();
         prefetch_tensor_map(&map_w);
@@ -472,6 +476,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     } else {
         // ================= epilogue warps =================
         const int q = warp & 3;        // tensor-memory lane quadrant this warp may read
+        constexpr int CW = BN / (Cfg::EW / 4);                   // columns (batch slots) of a tile this warp drains
+        const int c_begin = ((warp - 2 - Cfg::UW) >> 2) * CW;
         const int r = q * 32 + lane;   // feature row of the tile
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         uint32_t tile_it = 0;
@@ -487,12 +493,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if (!mbar_wait(tfull_bar(buf), (tile_it >> 1) & 1, a.status)) break;
             tcgen05_fence_after();
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = c_begin; c0 < c_begin + CW; c0 += 32) {
                 uint32_t u[32];
                 tmem_ld_x16(lane_addr + (uint32_t)(buf * BN + c0), *reinterpret_cast<uint32_t(*)[16]>(&u[0]));
                 tmem_ld_x16(lane_addr + (uint32_t)(buf * BN + c0 + 16), *reinterpret_cast<uint32_t(*)[16]>(&u[16]));
                 tmem_ld_wait();
-                if (c0 + 32 >= BN) {  // everything of this accumulator is in registers: hand it back
+                if (c0 + 32 >= c_begin + CW) {  // this warp's share of the accumulator is in registers: hand it back
                     tcgen05_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(buf));
